@@ -1,0 +1,157 @@
+/*
+ * fly_verify.h - C ABI of the FLy loose-verification step for NVIDIA B200 (sm_100a).
+ *
+ * One call verifies one speculative-decoding round for a batch of sequences:
+ * for each of the K+1 target-model logit rows of a sequence it computes the
+ * softmax entropy and the greedy token (Eq. 1, Eq. 5), compares the greedy
+ * tokens with the K draft tokens (Eq. 2), applies the entropy gate (Eq. 6) and
+ * the deferred-window rule (Eq. 8 - Eq. 11; Algorithm 1, steps 3 and 4) and
+ * writes the accepted-token count and the tokens to append.
+ *
+ * Conventions
+ *   - Every pointer marked "dev" is device memory of the handle's device, owned
+ *     by the caller; the library never frees or keeps it.  Pointers marked
+ *     "host" are host memory.
+ *   - Rows: sequence b, position i (1-based, 1..K+1) is row b*(K+1) + (i-1).
+ *     Position K+1 is the bonus position.
+ *   - fly_verify_run is asynchronous on the given CUDA stream, allocates
+ *     nothing and never synchronises the host with the device.
+ *   - No function throws, aborts or traps.  Misuse that the host can see is
+ *     reported by the return code before anything is launched; conditions that
+ *     depend on device data (non-finite logits, draft ids out of range) are
+ *     reported per row in row_flags.
+ */
+#ifndef FLY_VERIFY_H_
+#define FLY_VERIFY_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fly_verify fly_verify_t; /* opaque; owns scratch memory only */
+
+typedef enum {
+  FLY_OK = 0,
+  FLY_ERR_INVALID_ARG = 1, /* null pointer, size out of range, inconsistent arguments */
+  FLY_ERR_UNSUPPORTED = 2, /* a valid request this build cannot serve (alignment, W > K in carry mode, ...) */
+  FLY_ERR_CUDA = 3,        /* a CUDA runtime call failed; see fly_verify_last_cuda_error */
+  FLY_ERR_TIMEOUT = 4      /* a bounded device-side wait ran out (fused path) */
+} fly_status_t;
+
+typedef enum { FLY_F32 = 0, FLY_BF16 = 1 } fly_dtype_t;
+
+/* Unit of the gate threshold theta.  The paper thresholds the normalised
+ * entropy h = H / log|V| in [0,1] (Eq. 5, Eq. 6).  NATS compares H (natural
+ * log) with theta directly; NORMALIZED compares H with theta * log(vocab). */
+typedef enum { FLY_THETA_NATS = 0, FLY_THETA_NORMALIZED = 1 } fly_theta_unit_t;
+
+/* What happens to a Defer mismatch j whose window j+1..j+W does not fit in the
+ * round (j + W > K).  REJECT is the paper's rule (the paragraph after Eq. 9):
+ * the mismatch is rejected at once and no state crosses rounds.  CARRY is an
+ * extension: if positions j+1..K hold no mismatch the token is kept
+ * provisionally and the remaining j+W-K window slots are checked against the
+ * first draft positions of the next round; a mismatch there revokes it. */
+typedef enum { FLY_BOUNDARY_REJECT = 0, FLY_BOUNDARY_CARRY = 1 } fly_boundary_t;
+
+/* Deferred state of one sequence between rounds (CARRY only).
+ * pending      window slots still open at the start of the next round (0: none)
+ * rollback_len tokens appended since and including the provisionally kept mismatch
+ * correction   the target's own token at that mismatch
+ * The zero state is {0, 0, -1}. */
+typedef struct {
+  int32_t pending;
+  int32_t rollback_len;
+  int32_t correction;
+} fly_state_t;
+
+typedef struct {
+  int32_t device;           /* CUDA device ordinal */
+  int32_t max_batch;        /* largest B of any run, >= 1 */
+  int32_t max_k;            /* largest K of any run, 1..63 */
+  int32_t vocab;            /* |V| >= 1: row length of the logits */
+  fly_dtype_t logits_dtype; /* storage type of the logits */
+  int32_t hidden;           /* 0: logits path only.  > 0: hidden size of the fused LM-head path */
+} fly_verify_config_t;
+
+/* Creates a handle and its scratch memory (per-row partial states for rows
+ * that are split over several thread blocks).  host pointers.  On failure
+ * *out is NULL. */
+fly_status_t fly_verify_create(const fly_verify_config_t* config, fly_verify_t** out);
+
+/* Frees the scratch memory and the handle.  NULL is accepted. */
+fly_status_t fly_verify_destroy(fly_verify_t* handle);
+
+typedef struct {
+  int32_t B; /* sequences, 1..max_batch */
+  int32_t K; /* draft tokens per sequence, 1..max_k */
+
+  /* Logits path: dev [B, K+1, V] of logits_dtype, V contiguous, consecutive rows
+   * row_stride elements apart (row_stride >= V; 0 means V). */
+  const void* logits;
+  int64_t row_stride;
+
+  /* Fused LM-head path (logits == NULL): the logits are hidden x weight, formed
+   * in fp32 on the tensor cores and never stored.
+   * hidden: dev [B*(K+1), hidden] bf16 row-major.
+   * weight: dev [hidden, V] bf16 row-major (V contiguous). */
+  const void* hidden;
+  const void* weight;
+
+  const int32_t* draft; /* dev [B, K] draft tokens yhat_1..yhat_K */
+
+  double theta;                /* gate threshold (Eq. 6); +inf gives exact-match acceptance (Eq. 3) */
+  fly_theta_unit_t theta_unit;
+  int32_t W;                   /* window length >= 0 (Eq. 8) */
+  fly_boundary_t boundary;
+
+  const fly_state_t* state_in; /* dev [B] or NULL (= zero state); CARRY only */
+  fly_state_t* state_out;      /* dev [B]; required for CARRY, optional for REJECT (zero state written).
+                                  May alias state_in. */
+
+  int32_t* accept_len;    /* dev [B]: s in 1..K+1, tokens to append this round (Eq. 11) */
+  int32_t* rollback;      /* dev [B] or NULL: tokens to remove BEFORE appending (non-zero only when a
+                             carried deferral is revoked) */
+  int32_t* out_tokens;    /* dev [B, K+1]: first s entries valid, the rest -1 (Algorithm 1's concat lines) */
+  int32_t* target_argmax; /* dev [B, K+1] or NULL: y_i of Eq. 1, lowest index among equal maxima */
+  float* entropy;         /* dev [B, K+1] or NULL: H_i in nats (numerator of Eq. 5) */
+  uint32_t* row_flags;    /* dev [B, K+1] or NULL: bit 0 non-finite logit (NaN, +inf, or no finite entry);
+                             bit 1 draft id outside [0, V) (treated as a mismatch) */
+} fly_verify_args_t;
+
+/* Runs one verification step on `cuda_stream` (a cudaStream_t; NULL = default
+ * stream).  Exactly one of args->logits / (args->hidden, args->weight) is set.
+ * Returns FLY_OK once the work is enqueued. */
+fly_status_t fly_verify_run(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
+
+/* Convenience for callers that hold HOST buffers: the same step with every
+ * pointer in args a host pointer (state_in/state_out included).  Inputs are
+ * copied to device staging buffers owned by the handle, the step runs, results
+ * are copied back and the stream is synchronised before returning.  Host
+ * buffers should be page-locked for full copy bandwidth.  Logits path only. */
+fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
+
+/* Launch-shape control for tuning and tests: splits > 0 forces every row to be
+ * cut into that many pieces (each reduced by its own thread block); 0 restores
+ * the automatic choice.  Results do not depend on it beyond fp32 rounding. */
+fly_status_t fly_verify_set_splits(fly_verify_t* handle, int32_t splits);
+
+/* Measurement hook: selects which kernels fly_verify_run launches.  Bit 0: the
+ * row reduction (entropy/argmax partial states); bit 1: the acceptance scan.
+ * The default, 3, is the whole step; anything else leaves the outputs stale
+ * and exists only so that one kernel can be timed back to back. */
+fly_status_t fly_verify_set_stages(fly_verify_t* handle, int32_t stage_mask);
+
+/* Number of kernels the last fly_verify_run enqueued (for accounting). */
+int32_t fly_verify_last_launch_count(const fly_verify_t* handle);
+
+/* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
+int32_t fly_verify_last_cuda_error(const fly_verify_t* handle);
+
+const char* fly_status_string(fly_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLY_VERIFY_H_ */

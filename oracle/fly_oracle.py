@@ -328,11 +328,18 @@ def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
             if not (0 <= int(draft[b, i]) < V):
                 flags[b, i] |= FLAG_BAD_DRAFT
         delta = match_indicator(draft[b], y[b, :K])
+        # The paper does not treat invalid input.  Reading used by both sides: a
+        # flagged position counts as a mismatch that the gate never defers, so
+        # an invalid token id can never be emitted.
+        Hg = [(-math.inf if flags[b, i] else H[b, i]) for i in range(K)]
+        for i in range(K):
+            if flags[b, i]:
+                delta[i] = 0
         if boundary == "reject":
-            res = verify_round_paper(delta, H[b, :K], th, W, draft[b], y[b])
+            res = verify_round_paper(delta, Hg, th, W, draft[b], y[b])
         elif boundary == "carry":
             sin = ZERO_STATE if state_in is None else State(*[int(t) for t in state_in[b]])
-            res = verify_round_carry(delta, H[b, :K], th, W, draft[b], y[b], sin)
+            res = verify_round_carry(delta, Hg, th, W, draft[b], y[b], sin)
         else:
             raise ValueError(boundary)
         acc[b] = res.accept_len

@@ -1,0 +1,202 @@
+"""ctypes binding of the C ABI in include/fly_verify.h.
+
+Argument marshalling only: every step of the verification runs in the CUDA
+kernels of libfly_verify.so.  There is no CPU fallback; a missing library that
+cannot be built raises ImportError.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+from typing import Optional
+
+from . import build as _build
+
+FLY_OK, FLY_ERR_INVALID_ARG, FLY_ERR_UNSUPPORTED, FLY_ERR_CUDA, FLY_ERR_TIMEOUT = range(5)
+FLY_F32, FLY_BF16 = 0, 1
+FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
+FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
+
+EXPORTS = (
+    "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host",
+    "fly_verify_set_splits", "fly_verify_set_stages", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
+    "fly_status_string",
+)
+
+
+class fly_verify_config_t(C.Structure):
+    _fields_ = [("device", C.c_int32), ("max_batch", C.c_int32), ("max_k", C.c_int32),
+                ("vocab", C.c_int32), ("logits_dtype", C.c_int), ("hidden", C.c_int32)]
+
+
+class fly_verify_args_t(C.Structure):
+    _fields_ = [
+        ("B", C.c_int32), ("K", C.c_int32),
+        ("logits", C.c_void_p), ("row_stride", C.c_int64),
+        ("hidden", C.c_void_p), ("weight", C.c_void_p),
+        ("draft", C.c_void_p),
+        ("theta", C.c_double), ("theta_unit", C.c_int), ("W", C.c_int32), ("boundary", C.c_int),
+        ("state_in", C.c_void_p), ("state_out", C.c_void_p),
+        ("accept_len", C.c_void_p), ("rollback", C.c_void_p), ("out_tokens", C.c_void_p),
+        ("target_argmax", C.c_void_p), ("entropy", C.c_void_p), ("row_flags", C.c_void_p),
+    ]
+
+
+class FlyError(RuntimeError):
+    def __init__(self, status: int, what: str, cuda_error: int = 0):
+        self.status = status
+        self.cuda_error = cuda_error
+        super().__init__(f"{what}: {status_string(status)} (status {status}, cuda error {cuda_error})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads (building first if a source is newer) libfly_verify.so."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    try:
+        path = _build.ensure_built()
+        L = C.CDLL(path)
+    except Exception as e:  # no silent fallback: the CUDA library is the product
+        raise ImportError(f"libfly_verify.so is missing and could not be built: {e}") from e
+    L.fly_verify_create.argtypes = [C.POINTER(fly_verify_config_t), C.POINTER(C.c_void_p)]
+    L.fly_verify_create.restype = C.c_int
+    L.fly_verify_destroy.argtypes = [C.c_void_p]
+    L.fly_verify_destroy.restype = C.c_int
+    L.fly_verify_run.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p]
+    L.fly_verify_run.restype = C.c_int
+    L.fly_verify_run_host.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p]
+    L.fly_verify_run_host.restype = C.c_int
+    L.fly_verify_set_splits.argtypes = [C.c_void_p, C.c_int32]
+    L.fly_verify_set_splits.restype = C.c_int
+    L.fly_verify_set_stages.argtypes = [C.c_void_p, C.c_int32]
+    L.fly_verify_set_stages.restype = C.c_int
+    L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
+    L.fly_verify_last_launch_count.restype = C.c_int32
+    L.fly_verify_last_cuda_error.argtypes = [C.c_void_p]
+    L.fly_verify_last_cuda_error.restype = C.c_int32
+    L.fly_status_string.argtypes = [C.c_int]
+    L.fly_status_string.restype = C.c_char_p
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().fly_status_string(int(status)).decode()
+
+
+def _ptr(t) -> Optional[int]:
+    """Address of a torch tensor's storage (device or host), None for None."""
+    if t is None:
+        return None
+    return int(t.data_ptr())
+
+
+class FlyVerify:
+    """Handle of one verifier (fly_verify_create / fly_verify_destroy).
+
+    Tensors are torch tensors used purely as typed device (or, for run_host,
+    pinned host) buffers; the caller owns them.
+    """
+
+    def __init__(self, max_batch: int, max_k: int, vocab: int, dtype: str = "bf16", device: int = 0,
+                 hidden: int = 0):
+        self._h = C.c_void_p()
+        self.vocab = int(vocab)
+        self.dtype = dtype
+        cfg = fly_verify_config_t(int(device), int(max_batch), int(max_k), int(vocab),
+                                  FLY_BF16 if dtype == "bf16" else FLY_F32, int(hidden))
+        st = lib().fly_verify_create(C.byref(cfg), C.byref(self._h))
+        if st != FLY_OK:
+            self._h = C.c_void_p()
+            raise FlyError(st, "fly_verify_create")
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib().fly_verify_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_splits(self, splits: int):
+        st = lib().fly_verify_set_splits(self._h, int(splits))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_set_splits")
+
+    def set_stages(self, mask: int):
+        st = lib().fly_verify_set_stages(self._h, int(mask))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_set_stages")
+
+    @property
+    def last_launch_count(self) -> int:
+        return int(lib().fly_verify_last_launch_count(self._h))
+
+    def make_args(self, B, K, draft, accept_len, out_tokens, logits=None, row_stride=0, hidden=None,
+                  weight=None, theta=1.0, theta_unit="nats", W=3, boundary="reject", state_in=None,
+                  state_out=None, rollback=None, target_argmax=None, entropy=None, row_flags=None):
+        a = fly_verify_args_t()
+        a.B, a.K = int(B), int(K)
+        a.logits, a.row_stride = _ptr(logits), int(row_stride)
+        a.hidden, a.weight = _ptr(hidden), _ptr(weight)
+        a.draft = _ptr(draft)
+        a.theta = float(theta)
+        a.theta_unit = FLY_THETA_NATS if theta_unit == "nats" else FLY_THETA_NORMALIZED
+        a.W = int(W)
+        a.boundary = FLY_BOUNDARY_CARRY if boundary == "carry" else FLY_BOUNDARY_REJECT
+        a.state_in, a.state_out = _ptr(state_in), _ptr(state_out)
+        a.accept_len, a.rollback, a.out_tokens = _ptr(accept_len), _ptr(rollback), _ptr(out_tokens)
+        a.target_argmax, a.entropy, a.row_flags = _ptr(target_argmax), _ptr(entropy), _ptr(row_flags)
+        return a
+
+    def run(self, args: fly_verify_args_t, stream: int = 0):
+        """fly_verify_run: device buffers, asynchronous on `stream` (a raw cudaStream_t value)."""
+        st = lib().fly_verify_run(self._h, C.byref(args), C.c_void_p(stream))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_run", lib().fly_verify_last_cuda_error(self._h))
+
+    def run_host(self, args: fly_verify_args_t, stream: int = 0):
+        """fly_verify_run_host: host buffers, copies in and out, synchronises."""
+        st = lib().fly_verify_run_host(self._h, C.byref(args), C.c_void_p(stream))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_run_host", lib().fly_verify_last_cuda_error(self._h))
+
+
+class VerifyBuffers:
+    """Output buffers of one step, allocated once with torch and reused."""
+
+    def __init__(self, B: int, K: int, device, pinned: bool = False):
+        import torch
+        kw = dict(device=device)
+        if pinned:
+            kw = dict(device="cpu", pin_memory=True)
+        self.accept_len = torch.empty(B, dtype=torch.int32, **kw)
+        self.rollback = torch.empty(B, dtype=torch.int32, **kw)
+        self.out_tokens = torch.empty(B, K + 1, dtype=torch.int32, **kw)
+        self.target_argmax = torch.empty(B, K + 1, dtype=torch.int32, **kw)
+        self.entropy = torch.empty(B, K + 1, dtype=torch.float32, **kw)
+        self.row_flags = torch.empty(B, K + 1, dtype=torch.int32, **kw)
+        zero = torch.tensor([[0, 0, -1]] * B, dtype=torch.int32)   # the zero state of every sequence
+        self.state = zero.pin_memory() if pinned else zero.to(device)
+
+
+def verify(fv: FlyVerify, logits, draft, out: VerifyBuffers, theta=1.0, W=3, theta_unit="nats",
+           boundary="reject", stream: int = 0, host: bool = False):
+    """One verification step on logits [B, K+1, V] and draft [B, K] (int32).
+    In carry mode out.state is both the carried-in and the carried-out state."""
+    B, K1, V = logits.shape
+    assert V == fv.vocab and logits.stride(2) == 1 and logits.stride(0) == K1 * logits.stride(1)
+    carry = boundary == "carry"
+    a = fv.make_args(B, K1 - 1, draft, out.accept_len, out.out_tokens, logits=logits,
+                     row_stride=logits.stride(1), theta=theta, theta_unit=theta_unit, W=W, boundary=boundary,
+                     state_in=out.state if carry else None, state_out=out.state, rollback=out.rollback,
+                     target_argmax=out.target_argmax, entropy=out.entropy, row_flags=out.row_flags)
+    (fv.run_host if host else fv.run)(a, stream)
+    return out

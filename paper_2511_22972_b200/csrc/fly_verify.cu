@@ -1,0 +1,335 @@
+// Host side of the C ABI declared in include/fly_verify.h: argument checks,
+// launch-shape selection and kernel launches.  No torch types, no allocation
+// inside fly_verify_run.
+#include "fly_verify.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "fly_common.cuh"
+#include "reduce_kernel.cuh"
+#include "scan_kernel.cuh"
+
+namespace {
+
+constexpr int kMaxSplits = 32;
+constexpr int kMaxK = 63;
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    want = dev;
+  }
+  ~DeviceGuard() {
+    if (ok && prev != want) cudaSetDevice(prev);
+  }
+  int want = -1;
+};
+
+}  // namespace
+
+struct fly_verify {
+  fly_verify_config_t cfg;
+  int sm_count = 148;
+  int64_t max_rows = 0;
+  fly::Partial* partials = nullptr;  // [max_rows * kMaxSplits]
+  int forced_splits = 0;
+  int stages = 3;
+  int last_splits = 1;
+  int last_launches = 0;
+  int last_cuda_error = 0;
+  // staging for fly_verify_run_host (allocated on first use)
+  void* st_logits = nullptr;
+  size_t st_logits_bytes = 0;
+  int32_t* st_ints = nullptr;  // draft | state_in | state_out | accept | rollback | tokens | argmax | flags
+  float* st_entropy = nullptr;
+};
+
+namespace {
+
+fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
+  h->last_cuda_error = (int)e;
+  return FLY_ERR_CUDA;
+}
+
+int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
+  const int64_t resident = (int64_t)h->sm_count * (2048 / fly::kReduceThreads);  // one full wave of blocks
+  int64_t s = (row_bytes + 16384) / 32768;  // ~32 KB per unit
+  if (s < 1) s = 1;
+  if (rows * s < resident) {
+    // few rows: cut finer so that every SM has work, but keep >= 8 KB per unit
+    int64_t need = (resident + rows - 1) / rows;
+    int64_t fine = row_bytes / 8192;
+    if (fine < 1) fine = 1;
+    s = need < fine ? need : fine;
+    if (s < 1) s = 1;
+  }
+  if (s > kMaxSplits) s = kMaxSplits;
+  if (s > max_pieces) s = max_pieces;
+  if (s < 1) s = 1;
+  return (int)s;
+}
+
+template <typename T>
+cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_stride, int V, int64_t rows,
+                          int forced, fly::Partial* partials, cudaStream_t st, int* splits_out) {
+  constexpr int kE = fly::Seg<T>::kElems;
+  const bool vec = ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
+                   (V >= kE * 32);
+  const int64_t row_bytes = (int64_t)V * (int64_t)sizeof(T);
+  if (vec) {
+    const int nseg = V / kE;
+    int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, nseg);
+    if (splits > nseg) splits = nseg;
+    const int segs_per_split = (nseg + splits - 1) / splits;
+    *splits_out = splits;
+    const unsigned grid = (unsigned)(rows * splits);
+    fly::reduce_rows_vec<T, 4><<<grid, fly::kReduceThreads, 0, st>>>(static_cast<const T*>(logits), row_stride, V, nseg,
+                                                                     splits, segs_per_split, partials);
+  } else {
+    int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, (V + 31) / 32);
+    if (splits > V) splits = V;
+    const int elems_per_split = (V + splits - 1) / splits;
+    *splits_out = splits;
+    const unsigned grid = (unsigned)(rows * splits);
+    fly::reduce_rows_scalar<T, 4><<<grid, fly::kReduceThreads, 0, st>>>(static_cast<const T*>(logits), row_stride, V,
+                                                                        splits, elems_per_split, partials);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_scan(const fly::ScanParams& p, cudaStream_t st) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)((p.B + fly::kScanWarps - 1) / fly::kScanWarps));
+  cfg.blockDim = dim3(fly::kScanThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fly::scan_sequences, p);
+}
+
+fly_status_t check_args(const fly_verify* h, const fly_verify_args_t* a) {
+  if (!h || !a) return FLY_ERR_INVALID_ARG;
+  if (a->B < 1 || a->B > h->cfg.max_batch) return FLY_ERR_INVALID_ARG;
+  if (a->K < 1 || a->K > h->cfg.max_k) return FLY_ERR_INVALID_ARG;
+  if (!a->draft || !a->accept_len || !a->out_tokens) return FLY_ERR_INVALID_ARG;
+  if (a->W < 0) return FLY_ERR_INVALID_ARG;
+  if (std::isnan(a->theta)) return FLY_ERR_INVALID_ARG;
+  if (a->theta_unit != FLY_THETA_NATS && a->theta_unit != FLY_THETA_NORMALIZED) return FLY_ERR_INVALID_ARG;
+  if (a->boundary != FLY_BOUNDARY_REJECT && a->boundary != FLY_BOUNDARY_CARRY) return FLY_ERR_INVALID_ARG;
+  const bool has_logits = a->logits != nullptr;
+  const bool has_fused = a->hidden != nullptr || a->weight != nullptr;
+  if (has_logits == has_fused) return FLY_ERR_INVALID_ARG;
+  if (has_fused && (!a->hidden || !a->weight)) return FLY_ERR_INVALID_ARG;
+  if (has_logits && a->row_stride != 0 && a->row_stride < h->cfg.vocab) return FLY_ERR_INVALID_ARG;
+  if (a->boundary == FLY_BOUNDARY_CARRY) {
+    if (!a->state_out) return FLY_ERR_INVALID_ARG;
+    if (a->W > a->K) return FLY_ERR_UNSUPPORTED;
+  } else if (a->state_in) {
+    return FLY_ERR_INVALID_ARG;  // the paper's rule has no cross-round state
+  }
+  return FLY_OK;
+}
+
+float theta_to_nats(const fly_verify* h, const fly_verify_args_t* a) {
+  double th = a->theta;
+  if (a->theta_unit == FLY_THETA_NORMALIZED) th *= std::log((double)h->cfg.vocab);
+  return (float)th;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* fly_status_string(fly_status_t s) {
+  switch (s) {
+    case FLY_OK: return "ok";
+    case FLY_ERR_INVALID_ARG: return "invalid argument";
+    case FLY_ERR_UNSUPPORTED: return "unsupported request";
+    case FLY_ERR_CUDA: return "CUDA runtime error";
+    case FLY_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out) {
+  if (out) *out = nullptr;
+  if (!c || !out) return FLY_ERR_INVALID_ARG;
+  if (c->max_batch < 1 || c->max_k < 1 || c->max_k > kMaxK || c->vocab < 1 || c->hidden < 0 || c->device < 0)
+    return FLY_ERR_INVALID_ARG;
+  if (c->logits_dtype != FLY_F32 && c->logits_dtype != FLY_BF16) return FLY_ERR_INVALID_ARG;
+  if (c->hidden > 0) return FLY_ERR_UNSUPPORTED;  // fused LM-head path: not built yet
+  fly_verify* h = new (std::nothrow) fly_verify();
+  if (!h) return FLY_ERR_INVALID_ARG;
+  h->cfg = *c;
+  h->max_rows = (int64_t)c->max_batch * (c->max_k + 1);
+  DeviceGuard g(c->device);
+  if (!g.ok) { delete h; return FLY_ERR_CUDA; }
+  int sms = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+  if (e != cudaSuccess) { delete h; return FLY_ERR_CUDA; }
+  h->sm_count = sms > 0 ? sms : 148;
+  e = cudaMalloc(&h->partials, (size_t)h->max_rows * kMaxSplits * sizeof(fly::Partial));
+  if (e != cudaSuccess) { delete h; return FLY_ERR_CUDA; }
+  *out = h;
+  return FLY_OK;
+}
+
+fly_status_t fly_verify_destroy(fly_verify_t* h) {
+  if (!h) return FLY_OK;
+  DeviceGuard g(h->cfg.device);
+  if (g.ok) {
+    cudaFree(h->partials);
+    cudaFree(h->st_logits);
+    cudaFree(h->st_ints);
+    cudaFree(h->st_entropy);
+  }
+  delete h;
+  return FLY_OK;
+}
+
+fly_status_t fly_verify_set_splits(fly_verify_t* h, int32_t splits) {
+  if (!h || splits < 0 || splits > kMaxSplits) return FLY_ERR_INVALID_ARG;
+  h->forced_splits = splits;
+  return FLY_OK;
+}
+
+fly_status_t fly_verify_set_stages(fly_verify_t* h, int32_t mask) {
+  if (!h || mask < 1 || mask > 3) return FLY_ERR_INVALID_ARG;
+  h->stages = mask;
+  return FLY_OK;
+}
+
+int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
+int32_t fly_verify_last_cuda_error(const fly_verify_t* h) { return h ? h->last_cuda_error : 0; }
+
+fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* cuda_stream) {
+  fly_status_t s = check_args(h, a);
+  if (s != FLY_OK) return s;
+  if (!a->logits) return FLY_ERR_UNSUPPORTED;  // fused LM-head path: not built yet
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int V = h->cfg.vocab;
+  const int64_t rows = (int64_t)a->B * (a->K + 1);
+  const int64_t stride = a->row_stride ? a->row_stride : V;
+  h->last_launches = 0;
+
+  int splits = h->last_splits;
+  cudaError_t e;
+  if (h->stages & 1) {
+    if (h->cfg.logits_dtype == FLY_BF16)
+      e = launch_reduce<__nv_bfloat16>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits);
+    else
+      e = launch_reduce<float>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches++;
+    h->last_splits = splits;
+  }
+  if (!(h->stages & 2)) return FLY_OK;
+
+  fly::ScanParams p;
+  p.B = a->B; p.K = a->K; p.V = V; p.splits = splits;
+  p.partials = h->partials;
+  p.draft = a->draft;
+  p.theta_nats = theta_to_nats(h, a);
+  p.W = a->W > 64 ? 64 : a->W;
+  p.carry = a->boundary == FLY_BOUNDARY_CARRY;
+  p.state_in = reinterpret_cast<const int32_t*>(a->state_in);
+  p.state_out = reinterpret_cast<int32_t*>(a->state_out);
+  p.accept_len = a->accept_len;
+  p.rollback = a->rollback;
+  p.out_tokens = a->out_tokens;
+  p.target_argmax = a->target_argmax;
+  p.entropy = a->entropy;
+  p.row_flags = a->row_flags;
+  e = launch_scan(p, st);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->last_launches++;
+  return FLY_OK;
+}
+
+fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, void* cuda_stream) {
+  fly_status_t s = check_args(h, a);
+  if (s != FLY_OK) return s;
+  if (!a->logits) return FLY_ERR_UNSUPPORTED;
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int V = h->cfg.vocab;
+  const size_t esz = h->cfg.logits_dtype == FLY_BF16 ? 2 : 4;
+  const int64_t K1 = a->K + 1, B = a->B, rows = B * K1;
+  const int64_t stride = a->row_stride ? a->row_stride : V;
+  cudaError_t e;
+  if (!h->st_ints) {
+    // staging sized once for the largest run this handle allows
+    const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
+    const size_t ints = (size_t)(mb * (mk1 - 1) + 3 * mb + 3 * mb + mb + mb + 3 * mb * mk1);
+    if ((e = cudaMalloc(&h->st_ints, ints * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMalloc(&h->st_entropy, (size_t)(mb * mk1) * sizeof(float))) != cudaSuccess) return cuda_fail(h, e);
+  }
+  const size_t logit_bytes = (size_t)(((rows - 1) * stride + V)) * esz;
+  if (logit_bytes > h->st_logits_bytes) {
+    cudaFree(h->st_logits);
+    h->st_logits = nullptr;
+    h->st_logits_bytes = 0;
+    if ((e = cudaMalloc(&h->st_logits, logit_bytes)) != cudaSuccess) return cuda_fail(h, e);
+    h->st_logits_bytes = logit_bytes;
+  }
+  const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
+  int32_t* d_draft = h->st_ints;
+  int32_t* d_state_in = d_draft + mb * (mk1 - 1);
+  int32_t* d_state_out = d_state_in + 3 * mb;
+  int32_t* d_accept = d_state_out + 3 * mb;
+  int32_t* d_rollback = d_accept + mb;
+  int32_t* d_tokens = d_rollback + mb;
+  int32_t* d_argmax = d_tokens + mb * mk1;
+  int32_t* d_flags = d_argmax + mb * mk1;
+
+  if ((e = cudaMemcpyAsync(h->st_logits, a->logits, logit_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(h, e);
+  if ((e = cudaMemcpyAsync(d_draft, a->draft, (size_t)(B * a->K) * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(h, e);
+  if (a->state_in &&
+      (e = cudaMemcpyAsync(d_state_in, a->state_in, (size_t)B * 12, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(h, e);
+
+  fly_verify_args_t d = *a;
+  d.logits = h->st_logits;
+  d.draft = d_draft;
+  d.state_in = a->state_in ? reinterpret_cast<const fly_state_t*>(d_state_in) : nullptr;
+  d.state_out = a->state_out ? reinterpret_cast<fly_state_t*>(d_state_out) : nullptr;
+  d.accept_len = d_accept;
+  d.rollback = a->rollback ? d_rollback : nullptr;
+  d.out_tokens = d_tokens;
+  d.target_argmax = a->target_argmax ? d_argmax : nullptr;
+  d.entropy = a->entropy ? h->st_entropy : nullptr;
+  d.row_flags = a->row_flags ? reinterpret_cast<uint32_t*>(d_flags) : nullptr;
+  s = fly_verify_run(h, &d, cuda_stream);
+  if (s != FLY_OK) return s;
+
+  auto back = [&](void* dst, const void* src, size_t n) -> bool {
+    if (!dst) return true;
+    e = cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess;
+  };
+  if (!back(a->accept_len, d_accept, (size_t)B * 4) || !back(a->rollback, d_rollback, (size_t)B * 4) ||
+      !back(a->out_tokens, d_tokens, (size_t)rows * 4) || !back(a->target_argmax, d_argmax, (size_t)rows * 4) ||
+      !back(a->entropy, h->st_entropy, (size_t)rows * 4) || !back(a->row_flags, d_flags, (size_t)rows * 4) ||
+      !back(a->state_out, d_state_out, (size_t)B * 12))
+    return cuda_fail(h, e);
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(h, e);
+  return FLY_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,151 @@
+// Acceptance scan of the FLy verification step: one warp per sequence.
+//
+// Lanes first fold the per-unit Partials of "their" rows into entropy and
+// greedy token, then the warp forms the match bits Delta_i (Eq. 2) and the gate
+// bits [H_i >= theta] (Eq. 6) with ballots and walks the mismatch set J in
+// ascending order exactly as Algorithm 1 does (steps 3 and 4): Strict rejects,
+// Defer looks at the next W positions (Eq. 8, Eq. 9), a window that does not
+// fit in the round rejects (paper) or is carried to the next round (extension).
+// Finally the lanes write the tokens to append (Algorithm 1's concat lines).
+#pragma once
+#include "fly_common.cuh"
+
+namespace fly {
+
+constexpr int kScanThreads = 128;
+constexpr int kScanWarps = kScanThreads / 32;
+constexpr int kMaxRows = 64;  // K + 1 <= 64
+
+struct ScanParams {
+  int B, K, V;
+  int splits;
+  const Partial* partials;  // [B*(K+1), splits]
+  const int32_t* draft;     // [B, K]
+  float theta_nats;
+  int W;
+  int carry;                // 0: paper rule at the round boundary, 1: carry extension
+  const int32_t* state_in;  // [B, 3] or null
+  int32_t* state_out;       // [B, 3] or null
+  int32_t* accept_len;      // [B]
+  int32_t* rollback;        // [B] or null
+  int32_t* out_tokens;      // [B, K+1]
+  int32_t* target_argmax;   // [B, K+1] or null
+  float* entropy;           // [B, K+1] or null
+  uint32_t* row_flags;      // [B, K+1] or null
+};
+
+struct RoundOutcome {
+  int s;         // accepted-token count, 1..K+1
+  int rollback;  // tokens to remove first (revoked carry), else 0
+  int revoke;    // 1: out_tokens = [correction]
+  int st_pending, st_len, st_corr_pos;  // state_out; st_corr_pos = position j whose y_j is the correction (0: none)
+};
+
+// mism / defer: bit (i-1) set <=> position i is a mismatch / has H_i >= theta.
+__device__ __forceinline__ RoundOutcome decide_round(uint64_t mism, uint64_t defer, int K, int W, int carry,
+                                                     int pend_in, int len_in) {
+  RoundOutcome o;
+  o.s = K + 1; o.rollback = 0; o.revoke = 0; o.st_pending = 0; o.st_len = 0; o.st_corr_pos = 0;
+  if (carry && pend_in > 0) {
+    const uint64_t first_r = pend_in >= 64 ? ~0ull : ((1ull << pend_in) - 1ull);
+    if (mism & first_r) {  // a mismatch inside the carried window: revoke
+      o.s = 1; o.rollback = len_in; o.revoke = 1;
+      return o;
+    }
+  }
+  uint64_t rest = mism;
+  while (rest) {
+    const int j = __ffsll((long long)rest);  // 1-based position of the next mismatch
+    rest &= rest - 1;
+    if (!((defer >> (j - 1)) & 1ull)) { o.s = j; return o; }  // Strict
+    // positions j+1 .. min(j+W, K)  <->  bits j .. min(j+W,K)-1
+    const int hi = min(j + W, K);
+    const uint64_t upto_hi = hi >= 64 ? ~0ull : ((1ull << hi) - 1ull);
+    const uint64_t upto_j = (1ull << j) - 1ull;  // j <= K <= 63
+    const uint64_t later = mism & upto_hi & ~upto_j;
+    if (later == 0 && j + W <= K) continue;  // benign: keep the draft token
+    if (later == 0 && carry) {               // window leaves the round clean: carry it
+      o.s = K + 1; o.st_pending = j + W - K; o.st_len = K - j + 2; o.st_corr_pos = j;
+      return o;
+    }
+    o.s = j;
+    return o;
+  }
+  return o;
+}
+
+__global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
+  __shared__ int sm_y[kScanWarps][kMaxRows];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.x * kScanWarps + warp;
+  // every thread waits for the producer grid (row reduction) to complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (b >= p.B) return;
+  const int K = p.K, K1 = p.K + 1;
+
+  uint64_t mism = 0, defer = 0;
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int i = half * 32 + lane;  // 0-based row of this sequence
+    bool is_mism = false, is_defer = false;
+    if (i < K1) {
+      const int64_t row = (int64_t)b * K1 + i;
+      const Partial* pp = p.partials + row * p.splits;
+      Partial acc = pp[0];
+      for (int s = 1; s < p.splits; ++s) merge_partial(acc, pp[s]);
+      // entropy is non-negative; rounding may leave -1e-7 on a one-hot row
+      const float H = fmaxf(kLn2 * (log2f(acc.S) - acc.u / acc.S), 0.f);
+      uint32_t flag = 0;
+      if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx < -9.0e29f) flag |= kFlagNonFinite;
+      int y = acc.idx;
+      if (flag || y < 0 || y >= p.V) y = 0;  // keep every emitted id in range
+      sm_y[warp][i] = y;
+      if (i < K) {
+        const int d = p.draft[(int64_t)b * K + i];
+        if (d < 0 || d >= p.V) flag |= kFlagBadDraft;
+        is_mism = (d != y) || flag;
+        is_defer = (H >= p.theta_nats) && !flag;  // a flagged position is never kept
+      }
+      if (p.target_argmax) p.target_argmax[row] = y;
+      if (p.entropy) p.entropy[row] = H;
+      if (p.row_flags) p.row_flags[row] = flag;
+    }
+    const uint64_t mb = __ballot_sync(0xffffffffu, is_mism);
+    const uint64_t db = __ballot_sync(0xffffffffu, is_defer);
+    mism |= mb << (32 * half);
+    defer |= db << (32 * half);
+  }
+  __syncwarp();
+
+  int pend = 0, len = 0, corr = -1;
+  if (p.carry && p.state_in) {
+    pend = p.state_in[b * 3 + 0];
+    len = p.state_in[b * 3 + 1];
+    corr = p.state_in[b * 3 + 2];
+  }
+  __syncwarp();  // state_in may alias state_out: all lanes read before lane 0 writes
+  const RoundOutcome o = decide_round(mism, defer, K, p.W, p.carry, pend, len);
+
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int i = half * 32 + lane;
+    if (i < K1) {
+      int tok = -1;
+      if (o.revoke) tok = (i == 0) ? corr : -1;
+      else if (i < o.s - 1) tok = p.draft[(int64_t)b * K + i];
+      else if (i == o.s - 1) tok = sm_y[warp][i];
+      p.out_tokens[(int64_t)b * K1 + i] = tok;
+    }
+  }
+  if (lane == 0) {
+    p.accept_len[b] = o.s;
+    if (p.rollback) p.rollback[b] = o.rollback;
+    if (p.state_out) {
+      p.state_out[b * 3 + 0] = o.st_pending;
+      p.state_out[b * 3 + 1] = o.st_len;
+      p.state_out[b * 3 + 2] = o.st_corr_pos ? sm_y[warp][o.st_corr_pos - 1] : -1;
+    }
+  }
+}
+
+}  // namespace fly

@@ -114,15 +114,19 @@ def make_logits(w: Workload, step: int, device="cpu", setting=0,
 
     entropy_fn(rows[n, V]) -> entropy in nats [n] (supplied by the caller; the
     tests pass the fp64 oracle).  With it, a row whose entropy lies within
-    `guard` of the gate threshold is redrawn so that the gate decision is the
+    `guard` of the gate threshold (or of any threshold in a list) is redrawn so that the gate decision is the
     same in any reasonable precision.
     """
     x = _draw_rows(w, device, setting, step, 0)
     if entropy_fn is not None:
-        th = w.theta if theta_nats is None else theta_nats
+        ths = w.theta if theta_nats is None else theta_nats
+        ths = list(ths) if isinstance(ths, (list, tuple)) else [ths]
         for attempt in range(1, 8):
             H = torch.as_tensor(entropy_fn(x)).to("cpu", torch.float64)
-            bad = torch.nonzero((H - th).abs() < guard).flatten()
+            near = torch.zeros_like(H, dtype=torch.bool)
+            for th in ths:
+                near |= (H - th).abs() < guard
+            bad = torch.nonzero(near).flatten()
             if bad.numel() == 0:
                 break
             fresh = _draw_rows(w, device, setting, step, attempt)
@@ -153,7 +157,7 @@ def make_draft(w: Workload, step: int, top5: torch.Tensor, setting=0) -> torch.T
     B, K, V = w.B, w.K, w.V
     top = top5.view(B, K + 1, -1)[:, :K]
     u = torch.rand(B, K, generator=g, device=device)
-    near = torch.randint(1, 5, (B, K), generator=g, device=device)
+    near = torch.randint(1, 5, (B, K), generator=g, device=device).clamp_(max=top.shape[-1] - 1)
     anyv = torch.randint(0, V, (B, K), generator=g, device=device)
     p_arg, p_near, _ = w.draft_mix
     d = top[..., 0].clone()

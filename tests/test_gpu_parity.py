@@ -1,0 +1,212 @@
+"""Parity of the CUDA path (called through the C ABI) with the fp64 oracle:
+bit-exact argmax / accept lengths / tokens / state, entropy within 1e-4 nats."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fly_oracle as O
+from paper_2511_22972_b200 import FlyVerify, synthetic as S
+from tests._parity import assert_parity, check, draw, gpu_step, oracle_step
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def small(dtype, B, K, V, **kw):
+    base = S.TINY if dtype == "f32" else S.LLAMA3
+    return S.shrink(base, B=B, K=K, V=V, **kw)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 2, 7, 33, 257, 1000, 4097, 8200])
+def test_small_and_odd_vocabularies(dtype, V):
+    # below one warp slice, odd lengths (element-wise path), and just past a vector slice
+    for K in (1, 2, 4):
+        w = small(dtype, B=3, K=K, V=V)
+        fv = FlyVerify(w.B, K, V, dtype)
+        logits, draft = draw(w, step=K, guard=V > 1)
+        check(fv, logits, draft, theta=1.0 if V > 4 else 0.3, W=1, what=f"{dtype} V={V} K={K}")
+        fv.close()
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 128256), ("bf16", 152064), ("f32", 32000), ("bf16", 50257), ("f32", 50257)])
+@pytest.mark.parametrize("splits", [0, 1, 3, 8, 32])
+def test_row_splitting_does_not_change_results(dtype, V, splits):
+    # several slices per warp, a ragged last slice, every split count incl. ones that do not divide V
+    w = small(dtype, B=2, K=3, V=V)
+    fv = FlyVerify(w.B, w.K, V, dtype)
+    fv.set_splits(splits)
+    logits, draft = draw(w, step=1)
+    check(fv, logits, draft, theta=1.0, W=2, what=f"{dtype} V={V} splits={splits}")
+    fv.close()
+
+
+def test_ties_pick_the_lowest_index_across_lanes_warps_and_blocks():
+    V = 128256
+    w = small("bf16", B=1, K=7, V=V)
+    fv = FlyVerify(1, 7, V, "bf16")
+    logits, draft = draw(w, step=3, guard=False)
+    g = torch.Generator().manual_seed(5)
+    rows = logits.view(-1, V)
+    for r in range(rows.shape[0]):
+        top = rows[r].float().max().item() + 1.0
+        n = int(torch.randint(2, 9, (1,), generator=g))
+        where = torch.randint(0, V, (n,), generator=g)
+        if r == 0:
+            where = torch.tensor([V - 1, 7, 8])            # same 16-byte segment and the very last element
+        if r == 1:
+            where = torch.tensor([1024 * 8 + 3, 1024 * 8 * 5 + 3])   # different slices of one warp
+        rows[r, where.to(DEV)] = top
+    for splits in (0, 1, 5):
+        fv.set_splits(splits)
+        out = gpu_step(fv, logits, draft, 1.0, 3)
+        ref = oracle_step(logits, draft, 1.0, 3)
+        assert np.array_equal(out.target_argmax.cpu().numpy(), ref.target_argmax)
+    # bf16 rows of Gaussians tie at the top on their own
+    x = (torch.randn(64, V, generator=torch.Generator().manual_seed(1)) * 2).to(torch.bfloat16)
+    tied = (x.float() == x.float().max(dim=1, keepdim=True).values).sum(dim=1)
+    assert (tied > 1).any()
+    fv2 = FlyVerify(8, 7, V, "bf16")
+    lg = x.view(8, 8, V).to(DEV)
+    dr = torch.zeros(8, 7, dtype=torch.int32, device=DEV)
+    out = gpu_step(fv2, lg, dr, 1.0, 3)
+    ref = oracle_step(lg, dr, 1.0, 3)
+    assert np.array_equal(out.target_argmax.cpu().numpy(), ref.target_argmax)
+
+
+def test_masked_and_nonfinite_logits_and_bad_drafts():
+    V = 4096 + 24
+    w = small("bf16", B=6, K=3, V=V)
+    for dtype in ("bf16", "f32"):
+        w = small(dtype, B=6, K=3, V=V)
+        fv = FlyVerify(w.B, w.K, V, dtype)
+        logits, draft = draw(w, step=2, guard=False)
+        logits[0, 1, 100:3000] = -math.inf          # masked vocabulary range: allowed
+        logits[1, 0, 17] = math.nan
+        logits[2, 2, V - 1] = math.inf
+        logits[3, 3, :] = -math.inf                 # nothing finite
+        logits[4, 1, :] = -math.inf
+        logits[4, 1, 2000] = 0.5                    # one-hot: entropy exactly 0
+        draft[5, 0] = V                             # out of vocabulary
+        draft[5, 2] = -1
+        # redraw drafts of the masked rows against the edited logits
+        out = gpu_step(fv, logits, draft, 0.5, 1)
+        ref = oracle_step(logits, draft, 0.5, 1)
+        assert ref.row_flags[1, 0] == 1 and ref.row_flags[2, 2] == 1 and ref.row_flags[3, 3] == 1
+        assert ref.row_flags[5, 0] == 2 and ref.row_flags[5, 2] == 2 and ref.row_flags[0].sum() == 0
+        assert_parity(out, ref, dtype)
+        assert out.entropy[4, 1].item() == 0.0 and out.target_argmax[4, 1].item() == 2000
+        toks = out.out_tokens.cpu().numpy()
+        assert ((toks >= -1) & (toks < V)).all()     # nothing out of range is ever emitted
+        fv.close()
+
+
+def test_strided_rows_and_unaligned_base():
+    V = 5000
+    w = small("bf16", B=2, K=2, V=V)
+    logits, draft = draw(w, step=4)
+    fv = FlyVerify(2, 2, V, "bf16")
+    # rows 5008 elements apart (16-byte multiple): vector path with a stride
+    wide = torch.full((2, 3, 5008), 99.0, dtype=torch.bfloat16, device=DEV)
+    wide[:, :, :V] = logits
+    check(fv, wide[:, :, :V], draft, 1.0, 1, what="strided")
+    # base pointer off by one element: element-wise path
+    flat = torch.zeros(2 * 3 * V + 1, dtype=torch.bfloat16, device=DEV)
+    off = flat[1:].view(2, 3, V)
+    off.copy_(logits)
+    assert off.data_ptr() % 16 != 0
+    check(fv, off, draft, 1.0, 1, what="unaligned")
+
+
+def test_theta_units_and_limits():
+    V = 32000
+    w = small("f32", B=4, K=8, V=V)
+    fv = FlyVerify(4, 8, V, "f32")
+    th_norm = 0.3
+    logits, draft = draw(w, step=9, thetas=[th_norm * math.log(V), 1.0])
+    check(fv, logits, draft, th_norm, 3, theta_unit="normalized", what="normalized theta")
+    # theta = +inf: exact-match acceptance (Eq. 3)
+    _, out, ref = check(fv, logits, draft, math.inf, 3, what="theta=inf")
+    for b in range(4):
+        delta = O.match_indicator(draft[b].tolist(), ref.target_argmax[b, :8])
+        assert out.accept_len[b].item() == O.s_standard(delta)
+    # theta = 0, W = 0: everything accepted
+    _, out, _ = check(fv, logits, draft, 0.0, 0, what="theta=0 W=0")
+    assert (out.accept_len == 9).all()
+    # very long windows behave like W = K+1
+    check(fv, logits, draft, 1.0, 1000, what="W=1000")
+
+
+@pytest.mark.parametrize("K", [1, 15, 25, 31, 32, 47, 63])
+def test_draft_lengths_up_to_63(K):
+    V = 2048
+    w = small("bf16", B=5, K=K, V=V, draft_mix=(0.85, 0.1, 0.05))
+    fv = FlyVerify(5, K, V, "bf16")
+    logits, draft = draw(w, step=K, thetas=[0.5])
+    for W in (0, 1, 6, K):
+        check(fv, logits, draft, 0.5, W, what=f"K={K} W={W}")
+        check(fv, logits, draft, 0.5, W, boundary="carry", state=[[0, 0, -1]] * 5, what=f"carry K={K} W={W}")
+
+
+def test_carry_chain_many_rounds_reduced_vocab():
+    # the serving recipe at reduced V, state chained over 512 rounds
+    w = S.shrink(S.SERVING, B=32, K=8, V=4096)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    state_gpu = [[0, 0, -1]] * w.B
+    state_ref = np.array(state_gpu)
+    seen = {"pending": 0, "revoke": 0}
+    for rnd in range(512):
+        logits, draft = draw(w, step=rnd)
+        out = gpu_step(fv, logits, draft, w.theta, w.W, "carry", state_gpu)
+        ref = oracle_step(logits, draft, w.theta, w.W, "carry", state_ref)
+        assert_parity(out, ref, f"round {rnd}")
+        state_gpu = out.state.cpu().numpy()
+        state_ref = ref.state_out
+        seen["pending"] += int((ref.state_out[:, 0] > 0).sum())
+        seen["revoke"] += int((ref.rollback > 0).sum())
+    assert seen["pending"] > 50 and seen["revoke"] > 10      # the extension's branches were exercised
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = small("bf16", B=4, K=8, V=128256)
+    fv = FlyVerify(4, 8, w.V, "bf16")
+    logits, draft = draw(w, step=0)
+    _, out_d, ref = check(fv, logits, draft, 1.0, 3, what="device")
+    lh = logits.cpu().pin_memory()
+    dh = draft.cpu().pin_memory()
+    out_h = gpu_step(fv, lh, dh, 1.0, 3, host=True)
+    assert_parity(out_h, ref, "host")
+    assert torch.equal(out_h.entropy, out_d.entropy.cpu())
+
+
+def test_api_misuse_returns_error_codes():
+    from paper_2511_22972_b200 import FlyError, VerifyBuffers, binding as Bd
+    V = 1024
+    fv = FlyVerify(2, 4, V, "bf16")
+    logits = torch.zeros(2, 5, V, dtype=torch.bfloat16, device=DEV)
+    draft = torch.zeros(2, 4, dtype=torch.int32, device=DEV)
+    out = VerifyBuffers(2, 4, DEV)
+
+    def run(**kw):
+        base = dict(B=2, K=4, draft=draft, accept_len=out.accept_len, out_tokens=out.out_tokens, logits=logits,
+                    state_out=out.state)
+        base.update(kw)
+        fv.run(fv.make_args(**base))
+
+    run()
+    for bad, code in [(dict(B=3), Bd.FLY_ERR_INVALID_ARG), (dict(K=5), Bd.FLY_ERR_INVALID_ARG),
+                      (dict(B=0), Bd.FLY_ERR_INVALID_ARG), (dict(W=-1), Bd.FLY_ERR_INVALID_ARG),
+                      (dict(draft=None), Bd.FLY_ERR_INVALID_ARG), (dict(logits=None), Bd.FLY_ERR_INVALID_ARG),
+                      (dict(theta=math.nan), Bd.FLY_ERR_INVALID_ARG), (dict(row_stride=V - 8), Bd.FLY_ERR_INVALID_ARG),
+                      (dict(boundary="carry", W=5), Bd.FLY_ERR_UNSUPPORTED),
+                      (dict(boundary="carry", state_out=None), Bd.FLY_ERR_INVALID_ARG),
+                      (dict(state_in=out.state), Bd.FLY_ERR_INVALID_ARG)]:
+        with pytest.raises(FlyError) as e:
+            run(**bad)
+        assert e.value.status == code, bad
+    torch.cuda.synchronize()
+    run()                                                    # the handle is still usable
+    torch.cuda.synchronize()
+    assert fv.last_launch_count == 2

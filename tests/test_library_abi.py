@@ -1,0 +1,67 @@
+"""Host-side checks that need no GPU: the C-ABI library builds, loads and
+exports every symbol the header declares; argument errors are caught before
+any CUDA call."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2511_22972_b200 import binding as Bd, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "fly_verify.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fly_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_loads_and_exports_every_declared_symbol():
+    L = Bd.lib()
+    names = declared_symbols()
+    assert len(names) >= 8
+    for n in names:
+        assert hasattr(L, n), f"{n} is declared in the header but not exported"
+    assert sorted(Bd.EXPORTS) == names
+    assert os.path.exists(build.LIB_PATH) and not build.is_stale()
+
+
+def test_status_strings():
+    assert Bd.status_string(Bd.FLY_OK) == "ok"
+    assert "invalid" in Bd.status_string(Bd.FLY_ERR_INVALID_ARG)
+    assert "timed out" in Bd.status_string(Bd.FLY_ERR_TIMEOUT)
+    assert Bd.status_string(99) == "unknown status"
+
+
+def test_struct_layout_matches_the_header():
+    # x86-64 SysV: the args struct has 2 int32, then 8-byte members
+    assert C.sizeof(Bd.fly_verify_config_t) == 24
+    a = Bd.fly_verify_args_t
+    assert a.logits.offset == 8 and a.row_stride.offset == 16 and a.draft.offset == 40
+    assert a.theta.offset == 48 and a.theta_unit.offset == 56 and a.W.offset == 60 and a.boundary.offset == 64
+    assert a.state_in.offset == 72 and a.row_flags.offset == 128 and C.sizeof(a) == 136
+
+
+@pytest.mark.parametrize("cfg", [
+    dict(max_batch=0), dict(max_k=0), dict(max_k=64), dict(vocab=0), dict(dtype=7), dict(device=-1), dict(hidden=-1),
+])
+def test_create_rejects_bad_configs_without_touching_cuda(cfg):
+    base = dict(device=0, max_batch=4, max_k=8, vocab=1000, dtype=Bd.FLY_BF16, hidden=0)
+    base.update(cfg)
+    c = Bd.fly_verify_config_t(base["device"], base["max_batch"], base["max_k"], base["vocab"], base["dtype"],
+                               base["hidden"])
+    h = C.c_void_p(123)
+    st = Bd.lib().fly_verify_create(C.byref(c), C.byref(h))
+    assert st == Bd.FLY_ERR_INVALID_ARG and not h.value
+
+
+def test_null_arguments():
+    L = Bd.lib()
+    assert L.fly_verify_create(None, None) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_destroy(None) == Bd.FLY_OK
+    assert L.fly_verify_run(None, None, None) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_run_host(None, None, None) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_set_splits(None, 1) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_last_launch_count(None) == 0
