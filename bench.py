@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the FLy verification step (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path - row reduction (entropy, argmax),
+match/gate bits, deferred-window scan, token emission - over one batch of
+synthetic logits and draft tokens, through the C ABI.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1: launched by torch.distributed.run, one rank per GPU; every rank verifies
+its own B sequences (sequences are independent: weak scaling, no data-path
+collective) and the job time is the max over ranks.
+
+--impl reference times the fp64 CPU oracle (the only "reference implementation"
+of this method that exists here) on the host cores, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "loose-verify positions/s and HBM GB/s (% of B200 peak) at V=128256 bf16"
+UNIT = "positions/s"
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+L2_BYTES = 126 * 1024 * 1024
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-reduction kernel, from the ncu
+# captures summarised under profiles/ (bytes); None where no capture exists.
+NCU_TRAFFIC_BYTES = {
+}
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.sm.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+
+    def summary(self):
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.sm), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+def build_inputs(w, device, nbuf):
+    """nbuf distinct (logits, draft) pairs resident on the device.  No entropy guard here: timing does
+    not need gate decisions to be precision-proof (the parity tests draw guarded inputs)."""
+    import torch
+    from paper_2511_22972_b200 import synthetic as S
+    bufs = []
+    for i in range(nbuf):
+        logits = S.make_logits(w, i, device=device)
+        draft = S.make_draft(w, i, S.rank5(logits.view(-1, w.V)))
+        bufs.append((logits, draft))
+    torch.cuda.synchronize()
+    return bufs
+
+
+def time_steps(fv, arglist, stream, steps, warmup, ranks, launch):
+    """Device time of `steps` back-to-back steps: CUDA events on the launching stream, barrier and
+    synchronize on both sides, max over ranks.  Returns milliseconds for all steps."""
+    import torch
+    from paper_2511_22972_b200 import dist as D
+    n = len(arglist)
+    raw = stream.cuda_stream
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, 3)):
+            fv.run(arglist[i % n], raw)
+        graph, per_graph = None, 0
+        if launch == "graph":
+            per_graph = min(steps, 8 * n)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for i in range(per_graph):
+                    fv.run(arglist[i % n], raw)
+            graph.replay()
+        stream.synchronize()
+        D.barrier(ranks)
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        if graph is not None:
+            done = 0
+            while done < steps:
+                graph.replay()
+                done += per_graph
+            steps_run = done
+        else:
+            for i in range(steps):
+                fv.run(arglist[i % n], raw)
+            steps_run = steps
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        D.barrier(ranks)
+    ms = e0.elapsed_time(e1) * (steps / steps_run)
+    return D.max_over_ranks(ranks, ms)
+
+
+def oracle_rate(w, seconds_budget=12.0):
+    """The fp64 oracle as it stands, on this host's cores, on whole steps of the workload drawn by the
+    same generator, until the budget is used (at least one step, or a row sample if one step is too long)."""
+    import numpy as np
+    import torch
+    from oracle import fly_oracle as O
+    from paper_2511_22972_b200 import synthetic as S
+    torch.set_num_threads(1)
+    rows_done, t_used, steps = 0, 0.0, 0
+    B = w.B
+    # bound one sample to ~150 rows so that a single call stays within seconds
+    if w.rows > 160:
+        B = max(1, 160 // (w.K + 1))
+    ws = S.shrink(w, B=B)
+    while t_used < seconds_budget:
+        logits = S.make_logits(ws, steps, device="cpu")
+        draft = S.make_draft(ws, steps, S.rank5(logits.view(-1, ws.V)))
+        x = logits.double().numpy()
+        d = draft.numpy()
+        t0 = time.perf_counter()
+        O.verify_batch(x, d, w.theta, w.W, boundary=w.boundary,
+                       state_in=np.array([[0, 0, -1]] * ws.B) if w.boundary == "carry" else None)
+        t_used += time.perf_counter() - t0
+        rows_done += ws.rows
+        steps += 1
+    return rows_done / t_used, f"{steps} steps of {ws.B} sequences x {ws.K + 1} rows x V={ws.V} ({w.dtype} widened to fp64)", 1
+
+
+def run_reference(args, w):
+    """--impl reference: the oracle on the host cores; rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    from oracle import fly_oracle as O
+    from paper_2511_22972_b200 import synthetic as S
+    torch.set_num_threads(1)
+    B = max(1, min(w.B, 48 // (w.K + 1)))          # bounded sample of the workload per step
+    ws = S.shrink(w, B=B)
+
+    def one(step):
+        logits = S.make_logits(ws, step, device="cpu")
+        draft = S.make_draft(ws, step, S.rank5(logits.view(-1, ws.V)))
+        return logits.double().numpy(), draft.numpy()
+
+    data = [one(i) for i in range(min(4, args.steps + args.warmup))]
+    st = np.array([[0, 0, -1]] * ws.B) if w.boundary == "carry" else None
+    for i in range(args.warmup):
+        O.verify_batch(*data[i % len(data)], w.theta, w.W, boundary=w.boundary, state_in=st)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        O.verify_batch(*data[i % len(data)], w.theta, w.W, boundary=w.boundary, state_in=st)
+    dt = time.perf_counter() - t0
+    value = ws.rows * args.steps / dt
+    sample = f"each step = {ws.B} of {w.B} sequences ({ws.rows} rows x V={ws.V})"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype, "theta_nats": w.theta,
+                   "W": w.W, "boundary": w.boundary, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="llama3_vocab_batch")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--launch", default="stream", choices=["stream", "graph"])
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="plain stream order between steps (no programmatic dependent launch)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2511_22972_b200 import synthetic as S
+    w = S.WORKLOADS[args.workload]
+    if w.hidden:
+        raise SystemExit("the fused LM-head workload is not built yet")
+    if args.impl == "reference":
+        args.steps = args.steps or 5
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, w)
+        return
+    args.steps = args.steps or 20000
+    args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+
+    import torch
+    from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, dist as D
+    ranks = D.init_from_env("nccl")
+    assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
+    torch.cuda.set_device(ranks.local_rank)
+    device = torch.device("cuda", ranks.local_rank)
+    overlap = not args.no_overlap
+
+    step_bytes = w.rows * w.V * w.elem_bytes
+    nbuf = max(2, -(-int(2.4 * L2_BYTES) // step_bytes))     # rotate over > 2x L2 of distinct inputs
+    bufs = build_inputs(w, device, nbuf)
+    out = VerifyBuffers(w.B, w.K, device)
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype, device=ranks.local_rank)
+    fv.set_stream_overlap(overlap)
+    carry = w.boundary == "carry"
+    arglist = [fv.make_args(w.B, w.K, d, out.accept_len, out.out_tokens, logits=l, theta=w.theta, W=w.W,
+                            boundary=w.boundary, state_in=out.state if carry else None, state_out=out.state,
+                            rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
+                            row_flags=out.row_flags) for (l, d) in bufs]
+    stream = torch.cuda.Stream(device=device)
+
+    # ---- whole step, device-resident inputs --------------------------------------------------------
+    with ClockSampler(ranks.local_rank) as clk:
+        ms_total = time_steps(fv, arglist, stream, args.steps, args.warmup, ranks, args.launch)
+        launches_per_step = fv.last_launch_count
+        # ---- dominant kernel alone (row reduction), same buffers, same launch configuration ----------
+        fv.set_stages(1)
+        ms_reduce = time_steps(fv, arglist, stream, args.steps, 3, ranks, args.launch)
+        fv.set_stages(3)
+    ms_per_step = ms_total / args.steps
+    rows_all = w.rows * ranks.world
+    value = rows_all / (ms_per_step * 1e-3)
+
+    # ---- the same steps without cross-step overlap (plain stream order), for the record ---------------
+    fv.set_stream_overlap(False)
+    ms_serial = time_steps(fv, arglist, stream, max(args.steps // 4, 10), 3, ranks, args.launch) / max(args.steps // 4, 10)
+    fv.set_stream_overlap(overlap)
+
+    # ---- end to end through the host-buffer entry point ------------------------------------------------
+    e2e_steps = max(10, min(200, args.steps // 50))
+    host_l = [b[0].cpu().pin_memory() for b in bufs[:2]]
+    host_d = [b[1].cpu().pin_memory() for b in bufs[:2]]
+    hout = VerifyBuffers(w.B, w.K, device, pinned=True)
+    hargs = [fv.make_args(w.B, w.K, d, hout.accept_len, hout.out_tokens, logits=l, theta=w.theta, W=w.W,
+                          boundary=w.boundary, state_in=hout.state if carry else None, state_out=hout.state,
+                          rollback=hout.rollback, target_argmax=hout.target_argmax, entropy=hout.entropy,
+                          row_flags=hout.row_flags) for l, d in zip(host_l, host_d)]
+    raw = stream.cuda_stream
+    for i in range(3):
+        fv.run_host(hargs[i % 2], raw)
+    D.barrier(ranks)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        fv.run_host(hargs[i % 2], raw)          # synchronises the stream before returning
+    torch.cuda.synchronize()
+    e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
+    h2d = step_bytes + w.B * w.K * 4 + (w.B * 12 if carry else 0)
+    d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
+    e2e_value = rows_all * e2e_steps / e2e_s
+
+    peak, peak_kind = measured_hbm_peak()
+    achieved = step_bytes / (ms_reduce / args.steps * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
+                   "theta_nats": w.theta, "W": w.W, "boundary": w.boundary, "parallelism": f"dp{ranks.world}",
+                   "launch": args.launch, "stream_overlap": overlap,
+                   "l2": f"inputs rotate over {nbuf} distinct buffers = {nbuf * step_bytes / 1e6:.0f} MB (> 2x L2)"},
+        "hbm_gbs": rows_all * w.V * w.elem_bytes / (ms_per_step * 1e-3) / 1e9,
+        "hbm_pct_of_peak": 100.0 * step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+        "serialized": {"ms_per_step": ms_serial, "value": rows_all / (ms_serial * 1e-3),
+                       "note": "same steps in plain stream order (no overlap between consecutive steps)"},
+        "roofline": {"bound": "hbm", "kernel": "reduce_rows_vec (row reduction: entropy + argmax partial states)",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peak, "bytes_per_launch": step_bytes,
+                     "us_per_launch": ms_reduce / args.steps * 1e3,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "api": "fly_verify_run_host (pinned host buffers)"},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clk.summary(),
+    }
+    if ranks.is_main and ranks.world == 1 and not args.no_cpu_baseline:
+        v, sample, cores = oracle_rate(w)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    if ranks.is_main:
+        print(json.dumps(line), flush=True)
+    fv.close()
+    D.finalize(ranks)
+
+
+if __name__ == "__main__":
+    main()

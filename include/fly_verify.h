@@ -132,16 +132,30 @@ fly_status_t fly_verify_run(fly_verify_t* handle, const fly_verify_args_t* args,
  * buffers should be page-locked for full copy bandwidth.  Logits path only. */
 fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
 
-/* Launch-shape control for tuning and tests: splits > 0 forces every row to be
- * cut into that many pieces (each reduced by its own thread block); 0 restores
- * the automatic choice.  Results do not depend on it beyond fp32 rounding. */
-fly_status_t fly_verify_set_splits(fly_verify_t* handle, int32_t splits);
-
-/* Measurement hook: selects which kernels fly_verify_run launches.  Bit 0: the
- * row reduction (entropy/argmax partial states); bit 1: the acceptance scan.
- * The default, 3, is the whole step; anything else leaves the outputs stale
- * and exists only so that one kernel can be timed back to back. */
-fly_status_t fly_verify_set_stages(fly_verify_t* handle, int32_t stage_mask);
+/* Options of a handle (fly_verify_set_option).  None of them changes results
+ * beyond fp32 rounding order.
+ *
+ * FLY_OPT_SPLITS          > 0 forces every row to be cut into that many pieces (1..32), each reduced
+ *                         by its own thread block; 0 (default) chooses from the shape.
+ * FLY_OPT_SCAN_MODE       0 (default): the acceptance scan runs as the tail of the row-reduction
+ *                         kernel (the last block to finish a sequence's rows verifies it; one launch
+ *                         per step).  1: it runs as a kernel of its own (two launches per step).
+ * FLY_OPT_STAGES          measurement hook, bit 0 = row reduction, bit 1 = acceptance scan.  3 (default)
+ *                         is the whole step; 1 or 2 launch one kernel only (outputs are then stale or
+ *                         partial) so that it can be timed back to back.
+ * FLY_OPT_STREAM_OVERLAP  1: the row reduction is launched as a programmatic dependent of the
+ *                         previous kernel in the stream: it may start READING its logits while that
+ *                         kernel is still draining and waits for it to complete only before its
+ *                         first write.  Only correct if the logits of this step were complete
+ *                         before that previous kernel started (e.g. back-to-back steps over inputs
+ *                         already in memory).  0 (default): plain stream order. */
+typedef enum {
+  FLY_OPT_SPLITS = 0,
+  FLY_OPT_SCAN_MODE = 1,
+  FLY_OPT_STAGES = 2,
+  FLY_OPT_STREAM_OVERLAP = 3
+} fly_option_t;
+fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
 
 /* Number of kernels the last fly_verify_run enqueued (for accounting). */
 int32_t fly_verify_last_launch_count(const fly_verify_t* handle);

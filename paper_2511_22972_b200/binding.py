@@ -16,10 +16,11 @@ FLY_OK, FLY_ERR_INVALID_ARG, FLY_ERR_UNSUPPORTED, FLY_ERR_CUDA, FLY_ERR_TIMEOUT 
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
+FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STAGES, FLY_OPT_STREAM_OVERLAP = range(4)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host",
-    "fly_verify_set_splits", "fly_verify_set_stages", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
+    "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
 
@@ -70,10 +71,8 @@ def lib() -> C.CDLL:
     L.fly_verify_run.restype = C.c_int
     L.fly_verify_run_host.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p]
     L.fly_verify_run_host.restype = C.c_int
-    L.fly_verify_set_splits.argtypes = [C.c_void_p, C.c_int32]
-    L.fly_verify_set_splits.restype = C.c_int
-    L.fly_verify_set_stages.argtypes = [C.c_void_p, C.c_int32]
-    L.fly_verify_set_stages.restype = C.c_int
+    L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
+    L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
     L.fly_verify_last_launch_count.restype = C.c_int32
     L.fly_verify_last_cuda_error.argtypes = [C.c_void_p]
@@ -125,15 +124,22 @@ class FlyVerify:
         except Exception:
             pass
 
-    def set_splits(self, splits: int):
-        st = lib().fly_verify_set_splits(self._h, int(splits))
+    def set_option(self, option: int, value: int):
+        st = lib().fly_verify_set_option(self._h, int(option), int(value))
         if st != FLY_OK:
-            raise FlyError(st, "fly_verify_set_splits")
+            raise FlyError(st, "fly_verify_set_option")
+
+    def set_splits(self, splits: int):
+        self.set_option(FLY_OPT_SPLITS, splits)
+
+    def set_scan_mode(self, separate_kernel: bool):
+        self.set_option(FLY_OPT_SCAN_MODE, 1 if separate_kernel else 0)
 
     def set_stages(self, mask: int):
-        st = lib().fly_verify_set_stages(self._h, int(mask))
-        if st != FLY_OK:
-            raise FlyError(st, "fly_verify_set_stages")
+        self.set_option(FLY_OPT_STAGES, mask)
+
+    def set_stream_overlap(self, on: bool):
+        self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)
 
     @property
     def last_launch_count(self) -> int:

@@ -8,10 +8,13 @@ namespace fly {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-// Logits below this are treated as masked: they are clamped to it so that every
-// intermediate stays finite (a -inf logit has p = 0 and adds nothing to the
-// entropy; 0 * -inf would otherwise poison the weighted sum).
-constexpr float kMaskFloor = -1.0e30f;
+// Logits at or below this are treated as masked: they are clamped to it so that
+// every intermediate stays finite (a -inf logit has p = 0 and adds nothing to
+// the entropy; 0 * -inf would otherwise poison the weighted sum).  The value is
+// exactly representable in bf16 and small enough in magnitude that the rounding
+// of floor * log2(e) is negligible; a row whose maximum does not exceed it
+// counts as having no finite entry.
+constexpr float kMaskFloor = -999424.0f;
 constexpr int kIdxNone = 0x7fffffff;
 
 constexpr uint32_t kFlagNonFinite = 1u;

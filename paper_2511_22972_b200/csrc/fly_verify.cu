@@ -38,8 +38,11 @@ struct fly_verify {
   int sm_count = 148;
   int64_t max_rows = 0;
   fly::Partial* partials = nullptr;  // [max_rows * kMaxSplits]
+  unsigned int* tickets = nullptr;   // [max_batch], zero between launches
   int forced_splits = 0;
   int stages = 3;
+  int scan_mode = 0;   // 0: fused tail, 1: separate kernel
+  int overlap = 0;
   int last_splits = 1;
   int last_launches = 0;
   int last_cuda_error = 0;
@@ -57,27 +60,51 @@ fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
   return FLY_ERR_CUDA;
 }
 
+// Pieces per row.  Larger pieces amortise the per-block merge better, but the
+// grid needs enough blocks to fill every SM several times over and to divide
+// evenly among the SMs.  Among 1..32 take the smallest count whose blocks-per-SM
+// balance is within 3% of the best one, once there are >= 3.5 blocks per SM.
 int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
-  const int64_t resident = (int64_t)h->sm_count * (2048 / fly::kReduceThreads);  // one full wave of blocks
-  int64_t s = (row_bytes + 16384) / 32768;  // ~32 KB per unit
-  if (s < 1) s = 1;
-  if (rows * s < resident) {
-    // few rows: cut finer so that every SM has work, but keep >= 8 KB per unit
-    int64_t need = (resident + rows - 1) / rows;
-    int64_t fine = row_bytes / 8192;
-    if (fine < 1) fine = 1;
-    s = need < fine ? need : fine;
-    if (s < 1) s = 1;
+  const int64_t sms = h->sm_count;
+  int64_t cap = row_bytes / 8192;  // keep >= 8 KB per block
+  if (cap < 1) cap = 1;
+  if (cap > kMaxSplits) cap = kMaxSplits;
+  if (cap > max_pieces) cap = max_pieces;
+  double best = 0.0;
+  int64_t first_full = 0;
+  for (int64_t s = 1; s <= cap; ++s) {
+    const int64_t n = rows * s;
+    if (2 * n < 7 * sms) continue;
+    if (!first_full) first_full = s;
+    const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
+    if (bal > best) best = bal;
   }
-  if (s > kMaxSplits) s = kMaxSplits;
-  if (s > max_pieces) s = max_pieces;
-  if (s < 1) s = 1;
-  return (int)s;
+  if (!first_full) return (int)cap;  // tiny problem: as many blocks as allowed
+  for (int64_t s = first_full; s <= cap; ++s) {
+    const int64_t n = rows * s;
+    const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
+    if (bal >= best - 0.03) return (int)s;
+  }
+  return (int)cap;
+}
+
+void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned grid, unsigned block, cudaStream_t st,
+                 bool programmatic) {
+  memset(cfg, 0, sizeof(*cfg));
+  cfg->gridDim = dim3(grid);
+  cfg->blockDim = dim3(block);
+  cfg->dynamicSmemBytes = 0;
+  cfg->stream = st;
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = programmatic ? 1 : 0;
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
 }
 
 template <typename T>
 cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_stride, int V, int64_t rows,
-                          int forced, fly::Partial* partials, cudaStream_t st, int* splits_out) {
+                          int forced, fly::Partial* partials, cudaStream_t st, int* splits_out,
+                          fly::ScanParams tail, bool overlap) {
   constexpr int kE = fly::Seg<T>::kElems;
   const bool vec = ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
                    (V >= kE * 32);
@@ -88,33 +115,30 @@ cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_s
     if (splits > nseg) splits = nseg;
     const int segs_per_split = (nseg + splits - 1) / splits;
     *splits_out = splits;
-    const unsigned grid = (unsigned)(rows * splits);
-    fly::reduce_rows_vec<T, 4><<<grid, fly::kReduceThreads, 0, st>>>(static_cast<const T*>(logits), row_stride, V, nseg,
-                                                                     splits, segs_per_split, partials);
+    tail.splits = splits;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch(&cfg, attr, (unsigned)(rows * splits), fly::kReduceThreads, st, overlap);
+    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_vec<T, 4>, static_cast<const T*>(logits), row_stride, V, nseg,
+                              splits, segs_per_split, partials, tail);
   } else {
     int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, (V + 31) / 32);
     if (splits > V) splits = V;
     const int elems_per_split = (V + splits - 1) / splits;
     *splits_out = splits;
-    const unsigned grid = (unsigned)(rows * splits);
-    fly::reduce_rows_scalar<T, 4><<<grid, fly::kReduceThreads, 0, st>>>(static_cast<const T*>(logits), row_stride, V,
-                                                                        splits, elems_per_split, partials);
+    tail.splits = splits;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fill_launch(&cfg, attr, (unsigned)(rows * splits), fly::kReduceThreads, st, overlap);
+    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_scalar<T, 4>, static_cast<const T*>(logits), row_stride, V, splits,
+                              elems_per_split, partials, tail);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_scan(const fly::ScanParams& p, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = dim3((unsigned)((p.B + fly::kScanWarps - 1) / fly::kScanWarps));
-  cfg.blockDim = dim3(fly::kScanThreads);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  fill_launch(&cfg, attr, (unsigned)((p.B + fly::kScanWarps - 1) / fly::kScanWarps), fly::kScanThreads, st, true);
   return cudaLaunchKernelEx(&cfg, fly::scan_sequences, p);
 }
 
@@ -181,6 +205,9 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   h->sm_count = sms > 0 ? sms : 148;
   e = cudaMalloc(&h->partials, (size_t)h->max_rows * kMaxSplits * sizeof(fly::Partial));
   if (e != cudaSuccess) { delete h; return FLY_ERR_CUDA; }
+  e = cudaMalloc(&h->tickets, (size_t)c->max_batch * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(h->tickets, 0, (size_t)c->max_batch * sizeof(unsigned int));
+  if (e != cudaSuccess) { cudaFree(h->partials); cudaFree(h->tickets); delete h; return FLY_ERR_CUDA; }
   *out = h;
   return FLY_OK;
 }
@@ -190,6 +217,7 @@ fly_status_t fly_verify_destroy(fly_verify_t* h) {
   DeviceGuard g(h->cfg.device);
   if (g.ok) {
     cudaFree(h->partials);
+    cudaFree(h->tickets);
     cudaFree(h->st_logits);
     cudaFree(h->st_ints);
     cudaFree(h->st_entropy);
@@ -198,16 +226,27 @@ fly_status_t fly_verify_destroy(fly_verify_t* h) {
   return FLY_OK;
 }
 
-fly_status_t fly_verify_set_splits(fly_verify_t* h, int32_t splits) {
-  if (!h || splits < 0 || splits > kMaxSplits) return FLY_ERR_INVALID_ARG;
-  h->forced_splits = splits;
-  return FLY_OK;
-}
-
-fly_status_t fly_verify_set_stages(fly_verify_t* h, int32_t mask) {
-  if (!h || mask < 1 || mask > 3) return FLY_ERR_INVALID_ARG;
-  h->stages = mask;
-  return FLY_OK;
+fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v) {
+  if (!h) return FLY_ERR_INVALID_ARG;
+  switch (opt) {
+    case FLY_OPT_SPLITS:
+      if (v < 0 || v > kMaxSplits) return FLY_ERR_INVALID_ARG;
+      h->forced_splits = v;
+      return FLY_OK;
+    case FLY_OPT_SCAN_MODE:
+      if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
+      h->scan_mode = v;
+      return FLY_OK;
+    case FLY_OPT_STAGES:
+      if (v < 1 || v > 3) return FLY_ERR_INVALID_ARG;
+      h->stages = v;
+      return FLY_OK;
+    case FLY_OPT_STREAM_OVERLAP:
+      if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
+      h->overlap = v;
+      return FLY_OK;
+  }
+  return FLY_ERR_INVALID_ARG;
 }
 
 int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
@@ -225,22 +264,10 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   const int64_t stride = a->row_stride ? a->row_stride : V;
   h->last_launches = 0;
 
-  int splits = h->last_splits;
-  cudaError_t e;
-  if (h->stages & 1) {
-    if (h->cfg.logits_dtype == FLY_BF16)
-      e = launch_reduce<__nv_bfloat16>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits);
-    else
-      e = launch_reduce<float>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits);
-    if (e != cudaSuccess) return cuda_fail(h, e);
-    h->last_launches++;
-    h->last_splits = splits;
-  }
-  if (!(h->stages & 2)) return FLY_OK;
-
   fly::ScanParams p;
-  p.B = a->B; p.K = a->K; p.V = V; p.splits = splits;
+  p.B = a->B; p.K = a->K; p.V = V; p.splits = h->last_splits;
   p.partials = h->partials;
+  p.tickets = nullptr;
   p.draft = a->draft;
   p.theta_nats = theta_to_nats(h, a);
   p.W = a->W > 64 ? 64 : a->W;
@@ -253,9 +280,29 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   p.target_argmax = a->target_argmax;
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
-  e = launch_scan(p, st);
-  if (e != cudaSuccess) return cuda_fail(h, e);
-  h->last_launches++;
+
+  const bool fused_tail = h->stages == 3 && h->scan_mode == 0;
+  cudaError_t e;
+  if (h->stages & 1) {
+    fly::ScanParams tail = p;
+    tail.tickets = fused_tail ? h->tickets : nullptr;
+    int splits = 1;
+    if (h->cfg.logits_dtype == FLY_BF16)
+      e = launch_reduce<__nv_bfloat16>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
+                                       h->overlap != 0);
+    else
+      e = launch_reduce<float>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
+                               h->overlap != 0);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches++;
+    h->last_splits = splits;
+    p.splits = splits;
+  }
+  if ((h->stages & 2) && !fused_tail) {
+    e = launch_scan(p, st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches++;
+  }
   return FLY_OK;
 }
 

@@ -12,6 +12,7 @@
 // accumulations.
 #pragma once
 #include "fly_common.cuh"
+#include "scan_kernel.cuh"
 
 namespace fly {
 
@@ -91,7 +92,7 @@ template <int UNROLL>
 __device__ __forceinline__ void warp_slice_bf16(WarpAcc& a, const uint4* __restrict__ row, int seg0,
                                                 int seg_end, int lane) {
   constexpr uint32_t kNegInf2 = 0xff80ff80u;  // (-inf, -inf)
-  constexpr uint32_t kFloor2 = 0xf149f149u;   // bf16(-1e30) twice (0xf149 = -9.98e29)
+  constexpr uint32_t kFloor2 = 0xc974c974u;   // bf16(kMaskFloor) twice
   uint32_t w[UNROLL][4];
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j) {
@@ -241,13 +242,37 @@ __device__ __forceinline__ void block_finish(const WarpAcc& a, Partial* __restri
   }
 }
 
+// Fused tail: the block that completes a sequence's last unit verifies the
+// sequence.  Called by every thread after block_finish; only warp 0 acts.
+__device__ __forceinline__ void sequence_tail(const ScanParams& p, int row, int lane, int warp) {
+  __shared__ int sm_y[kMaxRows];
+  if (warp != 0 || p.tickets == nullptr) return;
+  const int K1 = p.K + 1;
+  const int b = row / K1;
+  unsigned last = 0;
+  if (lane == 0) {
+    __threadfence();  // the partial written above is visible before the ticket is taken
+    const unsigned t = atomicAdd(p.tickets + b, 1u);
+    last = (t == (unsigned)(K1 * p.splits) - 1u);
+    if (last) {
+      p.tickets[b] = 0;  // ready for the next launch
+      __threadfence();
+    }
+  }
+  last = __shfl_sync(0xffffffffu, last, 0);
+  if (last) {
+    __threadfence();  // every lane reads the other blocks' partials after the ticket was seen
+    scan_one_sequence(p, b, lane, sm_y);
+  }
+}
+
 // grid.x = rows * splits.  Vector path.
 //   segs_per_split  whole segments per unit (the last unit of a row may be short)
 //   nseg            whole segments in a row; elements [nseg*kElems, V) are the ragged tail
 template <typename T, int UNROLL>
 __global__ void __launch_bounds__(kReduceThreads)
 reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nseg, int splits, int segs_per_split,
-                Partial* __restrict__ partials) {
+                Partial* __restrict__ partials, const __grid_constant__ ScanParams tail) {
   constexpr int kE = Seg<T>::kElems;
   const int unit = blockIdx.x;
   const int row = unit / splits, split = unit - row * splits;
@@ -257,8 +282,9 @@ reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nse
   const int seg_begin = split * segs_per_split;
   const int seg_end = min(nseg, seg_begin + segs_per_split);
 
-  // Let the dependent scan kernel get scheduled; it waits for this grid's
-  // completion before it reads the partials.
+  // Let a programmatic dependent (the stand-alone scan kernel, or the next
+  // step's reduction) get scheduled; it waits for this grid's completion before
+  // it touches anything this grid writes.
   asm volatile("griddepcontrol.launch_dependents;");
 
   WarpAcc a;
@@ -271,14 +297,20 @@ reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nse
   // ragged tail (fewer than kElems logits): last unit of the row, last warp
   if (split == splits - 1 && warp == kReduceWarps - 1 && nseg * kE < V)
     warp_slice_scalar<T, 1>(a, rp, nseg * kE, V, lane);
+  // Everything above only reads the logits.  When this grid was launched as a
+  // programmatic dependent of the previous kernel in the stream, wait for that
+  // kernel to complete before the first write (scratch and outputs are shared
+  // between consecutive steps).  Otherwise this returns at once.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   block_finish(a, partials + unit, lane, warp);
+  sequence_tail(tail, row, lane, warp);
 }
 
 // grid.x = rows * splits.  Any alignment, any V.
 template <typename T, int UNROLL>
 __global__ void __launch_bounds__(kReduceThreads)
 reduce_rows_scalar(const T* __restrict__ logits, int64_t row_stride, int V, int splits, int elems_per_split,
-                   Partial* __restrict__ partials) {
+                   Partial* __restrict__ partials, const __grid_constant__ ScanParams tail) {
   const int unit = blockIdx.x;
   const int row = unit / splits, split = unit - row * splits;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -291,7 +323,9 @@ reduce_rows_scalar(const T* __restrict__ logits, int64_t row_stride, int V, int 
   constexpr int kSlice = UNROLL * 32;
   for (int e0 = e_begin + warp * kSlice; e0 < e_end; e0 += kReduceWarps * kSlice)
     warp_slice_scalar<T, UNROLL>(a, rp, e0, e_end, lane);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   block_finish(a, partials + unit, lane, warp);
+  sequence_tail(tail, row, lane, warp);
 }
 
 }  // namespace fly

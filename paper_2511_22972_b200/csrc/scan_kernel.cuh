@@ -1,4 +1,6 @@
-// Acceptance scan of the FLy verification step: one warp per sequence.
+// Acceptance scan of the FLy verification step: one warp per sequence.  It runs
+// either as the tail of the row-reduction kernel (the last block to finish a
+// sequence's rows does it) or as a launch of its own.
 //
 // Lanes first fold the per-unit Partials of "their" rows into entropy and
 // greedy token, then the warp forms the match bits Delta_i (Eq. 2) and the gate
@@ -20,6 +22,7 @@ struct ScanParams {
   int B, K, V;
   int splits;
   const Partial* partials;  // [B*(K+1), splits]
+  unsigned int* tickets;    // [B] arrival counters for the fused tail (zero between launches), or null
   const int32_t* draft;     // [B, K]
   float theta_nats;
   int W;
@@ -74,15 +77,17 @@ __device__ __forceinline__ RoundOutcome decide_round(uint64_t mism, uint64_t def
   return o;
 }
 
-__global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
-  __shared__ int sm_y[kScanWarps][kMaxRows];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int b = blockIdx.x * kScanWarps + warp;
-  // every thread waits for the producer grid (row reduction) to complete
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (b >= p.B) return;
-  const int K = p.K, K1 = p.K + 1;
+__device__ __forceinline__ Partial ld_partial_cg(const Partial* p) {
+  // partial states are written by other thread blocks: read them through L2
+  const int4 v = __ldcg(reinterpret_cast<const int4*>(p));
+  Partial q;
+  q.mx = __int_as_float(v.x); q.S = __int_as_float(v.y); q.u = __int_as_float(v.z); q.idx = v.w;
+  return q;
+}
 
+// One warp verifies sequence b.  sm_y: kMaxRows ints of shared memory private to the warp.
+__device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, int lane, int* sm_y) {
+  const int K = p.K, K1 = p.K + 1;
   uint64_t mism = 0, defer = 0;
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
@@ -91,15 +96,21 @@ __global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
     if (i < K1) {
       const int64_t row = (int64_t)b * K1 + i;
       const Partial* pp = p.partials + row * p.splits;
-      Partial acc = pp[0];
-      for (int s = 1; s < p.splits; ++s) merge_partial(acc, pp[s]);
+      Partial acc = empty_partial();
+      for (int s0 = 0; s0 < p.splits; s0 += 4) {  // four independent loads in flight
+        Partial q[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) q[t] = (s0 + t < p.splits) ? ld_partial_cg(pp + s0 + t) : empty_partial();
+#pragma unroll
+        for (int t = 0; t < 4; ++t) merge_partial(acc, q[t]);
+      }
       // entropy is non-negative; rounding may leave -1e-7 on a one-hot row
       const float H = fmaxf(kLn2 * (log2f(acc.S) - acc.u / acc.S), 0.f);
       uint32_t flag = 0;
-      if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx < -9.0e29f) flag |= kFlagNonFinite;
+      if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx <= kMaskFloor) flag |= kFlagNonFinite;
       int y = acc.idx;
       if (flag || y < 0 || y >= p.V) y = 0;  // keep every emitted id in range
-      sm_y[warp][i] = y;
+      sm_y[i] = y;
       if (i < K) {
         const int d = p.draft[(int64_t)b * K + i];
         if (d < 0 || d >= p.V) flag |= kFlagBadDraft;
@@ -133,7 +144,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
       int tok = -1;
       if (o.revoke) tok = (i == 0) ? corr : -1;
       else if (i < o.s - 1) tok = p.draft[(int64_t)b * K + i];
-      else if (i == o.s - 1) tok = sm_y[warp][i];
+      else if (i == o.s - 1) tok = sm_y[i];
       p.out_tokens[(int64_t)b * K1 + i] = tok;
     }
   }
@@ -143,9 +154,20 @@ __global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
     if (p.state_out) {
       p.state_out[b * 3 + 0] = o.st_pending;
       p.state_out[b * 3 + 1] = o.st_len;
-      p.state_out[b * 3 + 2] = o.st_corr_pos ? sm_y[warp][o.st_corr_pos - 1] : -1;
+      p.state_out[b * 3 + 2] = o.st_corr_pos ? sm_y[o.st_corr_pos - 1] : -1;
     }
   }
+}
+
+// Stand-alone launch: one warp per sequence, after the row reduction.
+__global__ void __launch_bounds__(kScanThreads) scan_sequences(ScanParams p) {
+  __shared__ int sm_y[kScanWarps][kMaxRows];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.x * kScanWarps + warp;
+  // every thread waits for the producer grid (row reduction) to complete
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (b >= p.B) return;
+  scan_one_sequence(p, b, lane, sm_y[warp]);
 }
 
 }  // namespace fly

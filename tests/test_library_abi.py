@@ -63,5 +63,5 @@ def test_null_arguments():
     assert L.fly_verify_destroy(None) == Bd.FLY_OK
     assert L.fly_verify_run(None, None, None) == Bd.FLY_ERR_INVALID_ARG
     assert L.fly_verify_run_host(None, None, None) == Bd.FLY_ERR_INVALID_ARG
-    assert L.fly_verify_set_splits(None, 1) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_set_option(None, 0, 1) == Bd.FLY_ERR_INVALID_ARG
     assert L.fly_verify_last_launch_count(None) == 0
