@@ -140,9 +140,6 @@ fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* 
  * FLY_OPT_SCAN_MODE       0 (default): the acceptance scan runs as the tail of the row-reduction
  *                         kernel (the last block to finish a sequence's rows verifies it; one launch
  *                         per step).  1: it runs as a kernel of its own (two launches per step).
- * FLY_OPT_STAGES          measurement hook, bit 0 = row reduction, bit 1 = acceptance scan.  3 (default)
- *                         is the whole step; 1 or 2 launch one kernel only (outputs are then stale or
- *                         partial) so that it can be timed back to back.
  * FLY_OPT_STREAM_OVERLAP  1: the row reduction is launched as a programmatic dependent of the
  *                         previous kernel in the stream: it may start READING its logits while that
  *                         kernel is still draining and waits for it to complete only before its
@@ -152,8 +149,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* 
 typedef enum {
   FLY_OPT_SPLITS = 0,
   FLY_OPT_SCAN_MODE = 1,
-  FLY_OPT_STAGES = 2,
-  FLY_OPT_STREAM_OVERLAP = 3
+  FLY_OPT_STREAM_OVERLAP = 2
 } fly_option_t;
 fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
 

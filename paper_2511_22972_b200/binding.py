@@ -16,7 +16,7 @@ FLY_OK, FLY_ERR_INVALID_ARG, FLY_ERR_UNSUPPORTED, FLY_ERR_CUDA, FLY_ERR_TIMEOUT 
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
-FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STAGES, FLY_OPT_STREAM_OVERLAP = range(4)
+FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host",
@@ -134,9 +134,6 @@ class FlyVerify:
 
     def set_scan_mode(self, separate_kernel: bool):
         self.set_option(FLY_OPT_SCAN_MODE, 1 if separate_kernel else 0)
-
-    def set_stages(self, mask: int):
-        self.set_option(FLY_OPT_STAGES, mask)
 
     def set_stream_overlap(self, on: bool):
         self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)

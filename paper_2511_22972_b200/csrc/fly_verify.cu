@@ -40,7 +40,6 @@ struct fly_verify {
   fly::Partial* partials = nullptr;  // [max_rows * kMaxSplits]
   unsigned int* tickets = nullptr;   // [max_batch], zero between launches
   int forced_splits = 0;
-  int stages = 3;
   int scan_mode = 0;   // 0: fused tail, 1: separate kernel
   int overlap = 0;
   int last_splits = 1;
@@ -237,10 +236,6 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->scan_mode = v;
       return FLY_OK;
-    case FLY_OPT_STAGES:
-      if (v < 1 || v > 3) return FLY_ERR_INVALID_ARG;
-      h->stages = v;
-      return FLY_OK;
     case FLY_OPT_STREAM_OVERLAP:
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->overlap = v;
@@ -281,9 +276,9 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
 
-  const bool fused_tail = h->stages == 3 && h->scan_mode == 0;
+  const bool fused_tail = h->scan_mode == 0;
   cudaError_t e;
-  if (h->stages & 1) {
+  {
     fly::ScanParams tail = p;
     tail.tickets = fused_tail ? h->tickets : nullptr;
     int splits = 1;
@@ -298,7 +293,7 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
     h->last_splits = splits;
     p.splits = splits;
   }
-  if ((h->stages & 2) && !fused_tail) {
+  if (!fused_tail) {
     e = launch_scan(p, st);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
