@@ -59,16 +59,24 @@ fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
   return FLY_ERR_CUDA;
 }
 
-// Pieces per row.  Larger pieces amortise the per-block merge better, but the
-// grid needs enough blocks to fill every SM several times over and to divide
-// evenly among the SMs.  Among 1..32 take the smallest count whose blocks-per-SM
+// Pieces per row.  Every block pays a fixed price (pipeline fill, block merge,
+// arrival ticket), so pieces should be large; but a grid that runs alone needs
+// enough blocks to fill every SM several times over and to divide evenly among
+// the SMs.  Among the allowed counts take the smallest whose blocks-per-SM
 // balance is within 3% of the best one, once there are >= 3.5 blocks per SM.
+// With stream overlap consecutive grids share the SMs, a single grid need not
+// fill the machine, and whole rows (or a few large pieces) are fastest.
 int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
   const int64_t sms = h->sm_count;
-  int64_t cap = row_bytes / 8192;  // keep >= 8 KB per block
+  int64_t cap = row_bytes / 32768;  // keep >= 32 KB per block
   if (cap < 1) cap = 1;
   if (cap > kMaxSplits) cap = kMaxSplits;
   if (cap > max_pieces) cap = max_pieces;
+  if (h->overlap) {
+    for (int64_t s = 1; s <= cap; ++s)
+      if (4 * rows * s >= sms) return (int)s;
+    return (int)cap;
+  }
   double best = 0.0;
   int64_t first_full = 0;
   for (int64_t s = 1; s <= cap; ++s) {
@@ -78,7 +86,7 @@ int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t ma
     const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
     if (bal > best) best = bal;
   }
-  if (!first_full) return (int)cap;  // tiny problem: as many blocks as allowed
+  if (!first_full) return (int)cap;  // small problem: as many blocks as allowed
   for (int64_t s = first_full; s <= cap; ++s) {
     const int64_t n = rows * s;
     const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
