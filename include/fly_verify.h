@@ -37,7 +37,8 @@ typedef enum {
   FLY_ERR_INVALID_ARG = 1, /* null pointer, size out of range, inconsistent arguments */
   FLY_ERR_UNSUPPORTED = 2, /* a valid request this build cannot serve (alignment, W > K in carry mode, ...) */
   FLY_ERR_CUDA = 3,        /* a CUDA runtime call failed; see fly_verify_last_cuda_error */
-  FLY_ERR_TIMEOUT = 4      /* a bounded device-side wait ran out (fused path) */
+  FLY_ERR_TIMEOUT = 4,     /* a bounded device-side wait ran out (fused path) */
+  FLY_ERR_TOO_LARGE = 5    /* fly_verify_run_static only: the step does not fit the built-in scratch area */
 } fly_status_t;
 
 typedef enum { FLY_F32 = 0, FLY_BF16 = 1 } fly_dtype_t;
@@ -131,6 +132,47 @@ fly_status_t fly_verify_run(fly_verify_t* handle, const fly_verify_args_t* args,
  * are copied back and the stream is synchronised before returning.  Host
  * buffers should be page-locked for full copy bandwidth.  Logits path only. */
 fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
+
+/* The paper has no counterpart of this entry point; it exists for callers that
+ * must not allocate device memory.
+ *
+ * Some hosts of this library cannot call cudaMalloc at the point where they
+ * verify: an inference server that has handed the whole device to its own
+ * memory pool, a plugin that runs inside another framework's execution
+ * callback, code that sits in a latency-critical loop where an allocation (an
+ * implicit device synchronisation) is not acceptable.  fly_verify_create
+ * allocates the scratch memory of a handle, so it is closed to them.  This
+ * function runs the same logits-path step (same kernels, same results) with NO
+ * handle: the per-piece partial states and the per-sequence arrival counters
+ * live in a fixed array that is part of the library image itself
+ * (FLY_STATIC_SCRATCH_BYTES of device memory on every GPU on which the library
+ * is loaded, held until the process exits).  It calls no cudaMalloc, cudaFree
+ * or other allocating routine.
+ *
+ *   device, vocab, logits_dtype   what fly_verify_config_t would carry
+ *   args                          as for fly_verify_run, device pointers, logits path only (hidden and
+ *                                 weight must be NULL); inputs and outputs are still the caller's
+ *
+ * Limits: B <= FLY_STATIC_MAX_BATCH, K <= 63 and B*(K+1) <= FLY_STATIC_MAX_PIECES.  Rows are cut into
+ * pieces as usual, but never into more than FLY_STATIC_MAX_PIECES pieces in total.  A step beyond the
+ * limits returns FLY_ERR_TOO_LARGE and launches nothing.
+ *
+ * The first call on each device looks up the device address of the built-in
+ * array (which also makes the CUDA runtime load the library's device code).
+ * Make that first call outside any stream capture; later calls only enqueue
+ * work on `cuda_stream` (one 4 KB memset of the arrival counters, one kernel).
+ *
+ * All calls on a device share the one array, and it keeps whatever the last
+ * call left there.  The counters are cleared on the stream at the start of
+ * every call and the partial states are fully rewritten before they are read,
+ * so stale contents never leak into a result.  But two calls whose work
+ * overlaps on the GPU (different streams, or several host threads) write the same
+ * scratch and corrupt each other: serialise them, e.g. keep them on one stream. */
+#define FLY_STATIC_MAX_BATCH 1024
+#define FLY_STATIC_MAX_PIECES 16384
+#define FLY_STATIC_SCRATCH_BYTES (FLY_STATIC_MAX_BATCH * 4 + FLY_STATIC_MAX_PIECES * 16) /* 260 KiB */
+fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t logits_dtype,
+                                   const fly_verify_args_t* args, void* cuda_stream);
 
 /* Options of a handle (fly_verify_set_option).  None of them changes results
  * beyond fp32 rounding order.

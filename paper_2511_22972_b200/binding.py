@@ -12,14 +12,15 @@ from typing import Optional
 
 from . import build as _build
 
-FLY_OK, FLY_ERR_INVALID_ARG, FLY_ERR_UNSUPPORTED, FLY_ERR_CUDA, FLY_ERR_TIMEOUT = range(5)
+FLY_OK, FLY_ERR_INVALID_ARG, FLY_ERR_UNSUPPORTED, FLY_ERR_CUDA, FLY_ERR_TIMEOUT, FLY_ERR_TOO_LARGE = range(6)
+FLY_STATIC_MAX_BATCH, FLY_STATIC_MAX_PIECES = 1024, 16384
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
 FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
-    "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host",
+    "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -71,6 +72,8 @@ def lib() -> C.CDLL:
     L.fly_verify_run.restype = C.c_int
     L.fly_verify_run_host.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p]
     L.fly_verify_run_host.restype = C.c_int
+    L.fly_verify_run_static.argtypes = [C.c_int32, C.c_int32, C.c_int, C.POINTER(fly_verify_args_t), C.c_void_p]
+    L.fly_verify_run_static.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -170,6 +173,22 @@ class FlyVerify:
         st = lib().fly_verify_run_host(self._h, C.byref(args), C.c_void_p(stream))
         if st != FLY_OK:
             raise FlyError(st, "fly_verify_run_host", lib().fly_verify_last_cuda_error(self._h))
+
+
+def run_static(args: fly_verify_args_t, vocab: int, dtype: str = "bf16", device: int = 0, stream: int = 0):
+    """fly_verify_run_static: the logits-path step without a handle, for callers that must not allocate
+    device memory (its scratch is a fixed array inside the library).  `args` is the same struct that
+    FlyVerify.run takes; `static_args` fills one without needing a handle.  Calls on one device must not
+    overlap on the GPU."""
+    st = lib().fly_verify_run_static(int(device), int(vocab), FLY_BF16 if dtype == "bf16" else FLY_F32,
+                                     C.byref(args), C.c_void_p(stream))
+    if st != FLY_OK:
+        raise FlyError(st, "fly_verify_run_static")
+
+
+def static_args(*a, **kw) -> fly_verify_args_t:
+    """Fills a fly_verify_args_t (same parameters as FlyVerify.make_args) without creating a handle."""
+    return FlyVerify.make_args(None, *a, **kw)
 
 
 class VerifyBuffers:

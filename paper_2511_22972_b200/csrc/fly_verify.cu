@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "fly_common.cuh"
@@ -189,6 +190,8 @@ const char* fly_status_string(fly_status_t s) {
     case FLY_ERR_UNSUPPORTED: return "unsupported request";
     case FLY_ERR_CUDA: return "CUDA runtime error";
     case FLY_ERR_TIMEOUT: return "device-side wait timed out";
+    case FLY_ERR_TOO_LARGE:
+      return "step exceeds the built-in scratch area (B <= 1024, B*(K+1) <= 16384)";
   }
   return "unknown status";
 }
@@ -380,6 +383,107 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     return cuda_fail(h, e);
   if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(h, e);
   return FLY_OK;
+}
+
+// ---------------------------------------------------------------------------
+// fly_verify_run_static: the logits-path step for callers that cannot allocate.
+// Its scratch is this array in the library image.  In host code the array's
+// name is only a handle for the runtime, not a device address: the address is
+// looked up once per device with cudaGetSymbolAddress and handed to the kernel
+// like any other scratch pointer.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_fly_static_scratch[FLY_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticSlot {
+  void* base = nullptr;  // device address of g_fly_static_scratch on this device
+  int sm_count = 0;
+};
+StaticSlot g_static_slots[kStaticMaxDevices];
+std::mutex g_static_mu;
+
+// Once per device, with that device current.
+cudaError_t static_scratch_for(int device, StaticSlot* out) {
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  StaticSlot& s = g_static_slots[device];
+  if (!s.base) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_fly_static_scratch);
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return e;
+    s.sm_count = sms > 0 ? sms : 148;
+    s.base = p;
+  }
+  *out = s;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t logits_dtype,
+                                   const fly_verify_args_t* a, void* cuda_stream) {
+  if (!a || device < 0 || device >= kStaticMaxDevices || vocab < 1) return FLY_ERR_INVALID_ARG;
+  if (logits_dtype != FLY_F32 && logits_dtype != FLY_BF16) return FLY_ERR_INVALID_ARG;
+  if (a->B > FLY_STATIC_MAX_BATCH && a->K >= 1 && a->K <= kMaxK) return FLY_ERR_TOO_LARGE;
+  fly_verify h;  // a stack stand-in for a handle: describes the step, owns nothing
+  h.cfg.device = device;
+  h.cfg.max_batch = FLY_STATIC_MAX_BATCH;
+  h.cfg.max_k = kMaxK;
+  h.cfg.vocab = vocab;
+  h.cfg.logits_dtype = logits_dtype;
+  h.cfg.hidden = 0;
+  fly_status_t s = check_args(&h, a);
+  if (s != FLY_OK) return s;
+  if (!a->logits) return FLY_ERR_UNSUPPORTED;  // the fused LM-head path needs a handle
+  const int64_t rows = (int64_t)a->B * (a->K + 1);
+  if (rows > FLY_STATIC_MAX_PIECES) return FLY_ERR_TOO_LARGE;
+
+  DeviceGuard g(device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  StaticSlot slot;
+  if (static_scratch_for(device, &slot) != cudaSuccess) return FLY_ERR_CUDA;
+  unsigned int* tickets = static_cast<unsigned int*>(slot.base);
+  fly::Partial* partials =
+      reinterpret_cast<fly::Partial*>(static_cast<unsigned char*>(slot.base) + FLY_STATIC_MAX_BATCH * 4);
+  h.sm_count = slot.sm_count;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t stride = a->row_stride ? a->row_stride : vocab;
+  const int64_t esz = logits_dtype == FLY_BF16 ? 2 : 4;
+  int splits = auto_splits(&h, rows, (int64_t)vocab * esz, kMaxSplits);
+  const int64_t room = FLY_STATIC_MAX_PIECES / rows;  // >= 1
+  if (splits > room) splits = (int)room;
+
+  fly::ScanParams p;
+  p.B = a->B; p.K = a->K; p.V = vocab; p.splits = splits;
+  p.partials = partials;
+  p.tickets = tickets;
+  p.draft = a->draft;
+  p.theta_nats = theta_to_nats(&h, a);
+  p.W = a->W > 64 ? 64 : a->W;
+  p.carry = a->boundary == FLY_BOUNDARY_CARRY;
+  p.state_in = reinterpret_cast<const int32_t*>(a->state_in);
+  p.state_out = reinterpret_cast<int32_t*>(a->state_out);
+  p.accept_len = a->accept_len;
+  p.rollback = a->rollback;
+  p.out_tokens = a->out_tokens;
+  p.target_argmax = a->target_argmax;
+  p.entropy = a->entropy;
+  p.row_flags = a->row_flags;
+
+  // The arrival counters must start at zero, whatever an earlier call left behind.
+  cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4, st);
+  if (e != cudaSuccess) return FLY_ERR_CUDA;
+  int used = 1;
+  if (logits_dtype == FLY_BF16)
+    e = launch_reduce<__nv_bfloat16>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
+  else
+    e = launch_reduce<float>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
+  return e == cudaSuccess ? FLY_OK : FLY_ERR_CUDA;
 }
 
 }  // extern "C"
