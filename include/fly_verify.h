@@ -93,10 +93,14 @@ typedef struct {
   const void* logits;
   int64_t row_stride;
 
-  /* Fused LM-head path (logits == NULL): the logits are hidden x weight, formed
-   * in fp32 on the tensor cores and never stored.
-   * hidden: dev [B*(K+1), hidden] bf16 row-major.
-   * weight: dev [hidden, V] bf16 row-major (V contiguous). */
+  /* Fused LM-head path (logits == NULL; the handle was created with hidden > 0):
+   * the logits are hidden x weight - the last linear layer of the target forward
+   * pass that yields l_1..l_{K+1} (Section 2.1) - formed in fp32 on the tensor
+   * cores and never stored.
+   * hidden: dev [B*(K+1), hidden] bf16 row-major, 16-byte aligned.
+   * weight: dev [hidden, V] bf16 row-major (V contiguous), 16-byte aligned.
+   * hidden and V must be multiples of 8 (fly_verify_create checks).  Positions
+   * are processed 288 at a time; each block of 288 streams the weight once. */
   const void* hidden;
   const void* weight;
 
@@ -130,7 +134,9 @@ fly_status_t fly_verify_run(fly_verify_t* handle, const fly_verify_args_t* args,
  * pointer in args a host pointer (state_in/state_out included).  Inputs are
  * copied to device staging buffers owned by the handle, the step runs, results
  * are copied back and the stream is synchronised before returning.  Host
- * buffers should be page-locked for full copy bandwidth.  Logits path only. */
+ * buffers should be page-locked for full copy bandwidth.  On the fused path
+ * hidden is a host pointer; weight (a model parameter, not a per-step input)
+ * remains a DEVICE pointer. */
 fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
 
 /* The paper has no counterpart of this entry point; it exists for callers that
@@ -194,6 +200,14 @@ typedef enum {
   FLY_OPT_STREAM_OVERLAP = 2
 } fly_option_t;
 fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
+
+/* The fused path's kernel waits on hardware barriers (TMA arrival, tensor-core
+ * completion); every such wait is bounded.  If one runs out, the kernel records
+ * it and returns without hanging (its outputs are then undefined).  This call
+ * synchronises `cuda_stream` and returns FLY_ERR_TIMEOUT if that happened since
+ * the last call (the record is cleared), else FLY_OK.  While a record is
+ * pending, further fused steps give up early.  Logits-path kernels have no waits. */
+fly_status_t fly_verify_device_status(fly_verify_t* handle, void* cuda_stream);
 
 /* Number of kernels the last fly_verify_run enqueued (for accounting). */
 int32_t fly_verify_last_launch_count(const fly_verify_t* handle);

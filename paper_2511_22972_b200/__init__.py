@@ -4,4 +4,4 @@
 `synthetic` draws the benchmark inputs; `build` compiles the library.
 """
 from . import binding, build, synthetic  # noqa: F401
-from .binding import FlyError, FlyVerify, VerifyBuffers, verify  # noqa: F401
+from .binding import FlyError, FlyVerify, VerifyBuffers, verify, verify_fused  # noqa: F401

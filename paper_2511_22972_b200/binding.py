@@ -21,6 +21,7 @@ FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
+    "fly_verify_device_status",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -74,6 +75,8 @@ def lib() -> C.CDLL:
     L.fly_verify_run_host.restype = C.c_int
     L.fly_verify_run_static.argtypes = [C.c_int32, C.c_int32, C.c_int, C.POINTER(fly_verify_args_t), C.c_void_p]
     L.fly_verify_run_static.restype = C.c_int
+    L.fly_verify_device_status.argtypes = [C.c_void_p, C.c_void_p]
+    L.fly_verify_device_status.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -140,6 +143,10 @@ class FlyVerify:
 
     def set_stream_overlap(self, on: bool):
         self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)
+
+    def device_status(self, stream: int = 0) -> int:
+        """fly_verify_device_status: synchronises the stream; FLY_OK or FLY_ERR_TIMEOUT."""
+        return int(lib().fly_verify_device_status(self._h, C.c_void_p(stream)))
 
     @property
     def last_launch_count(self) -> int:
@@ -220,5 +227,23 @@ def verify(fv: FlyVerify, logits, draft, out: VerifyBuffers, theta=1.0, W=3, the
                      row_stride=logits.stride(1), theta=theta, theta_unit=theta_unit, W=W, boundary=boundary,
                      state_in=out.state if carry else None, state_out=out.state, rollback=out.rollback,
                      target_argmax=out.target_argmax, entropy=out.entropy, row_flags=out.row_flags)
+    (fv.run_host if host else fv.run)(a, stream)
+    return out
+
+
+def verify_fused(fv: FlyVerify, hidden, weight, draft, out: VerifyBuffers, theta=1.0, W=3, theta_unit="nats",
+                 boundary="reject", stream: int = 0, host: bool = False):
+    """One verification step on the fused LM-head path: hidden [B*(K+1), D] bf16 and weight [D, V] bf16
+    (device; with host=True hidden, draft and the outputs are host buffers, the weight stays on the device).
+    The logits hidden @ weight are formed and reduced inside the kernel and never stored."""
+    B, K = draft.shape
+    rows, D = hidden.shape
+    assert rows == B * (K + 1) and tuple(weight.shape) == (D, fv.vocab)
+    assert hidden.is_contiguous() and weight.is_contiguous()
+    carry = boundary == "carry"
+    a = fv.make_args(B, K, draft, out.accept_len, out.out_tokens, hidden=hidden, weight=weight, theta=theta,
+                     theta_unit=theta_unit, W=W, boundary=boundary, state_in=out.state if carry else None,
+                     state_out=out.state, rollback=out.rollback, target_argmax=out.target_argmax,
+                     entropy=out.entropy, row_flags=out.row_flags)
     (fv.run_host if host else fv.run)(a, stream)
     return out

@@ -9,7 +9,10 @@
 #include <mutex>
 #include <new>
 
+#include <cudaTypedefs.h>
+
 #include "fly_common.cuh"
+#include "lmhead_kernel.cuh"
 #include "reduce_kernel.cuh"
 #include "scan_kernel.cuh"
 
@@ -46,6 +49,16 @@ struct fly_verify {
   int last_splits = 1;
   int last_launches = 0;
   int last_cuda_error = 0;
+  // fused LM-head path (cfg.hidden > 0)
+  fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]
+  int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
+  PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
+  CUtensorMap map_w, map_h;             // cached for (map_w_ptr, map_h_ptr, map_h_rows)
+  const void* map_w_ptr = nullptr;
+  const void* map_h_ptr = nullptr;
+  int64_t map_h_rows = 0;
+  void* st_hidden = nullptr;            // staging of fly_verify_run_host
+  size_t st_hidden_bytes = 0;
   // staging for fly_verify_run_host (allocated on first use)
   void* st_logits = nullptr;
   size_t st_logits_bytes = 0;
@@ -173,10 +186,88 @@ fly_status_t check_args(const fly_verify* h, const fly_verify_args_t* a) {
   return FLY_OK;
 }
 
+fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, const fly::Partial* partials, int splits);
+
+// 2-D bf16 tensor map with the 128-byte swizzle: dims {inner, outer}, row pitch in bytes, box {64, box_rows}.
+bool encode_map(fly_verify* h, CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                uint32_t box_rows) {
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = h->encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box,
+                                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Fused LM-head step: one GEMM + row-statistics launch per block of up to 288
+// positions, then the acceptance scan over the per-CTA partial states.
+fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t st) {
+  namespace L = fly::lmhead;
+  const int V = h->cfg.vocab, D = h->cfg.hidden;
+  const int64_t rows = (int64_t)a->B * (a->K + 1);
+  if ((reinterpret_cast<uintptr_t>(a->hidden) & 15u) || (reinterpret_cast<uintptr_t>(a->weight) & 15u))
+    return FLY_ERR_UNSUPPORTED;  // TMA needs 16-byte aligned bases
+  if (h->map_w_ptr != a->weight) {
+    if (!encode_map(h, &h->map_w, a->weight, (uint64_t)V, (uint64_t)D, (uint64_t)V * 2, 64)) return FLY_ERR_CUDA;
+    h->map_w_ptr = a->weight;
+  }
+  if (h->map_h_ptr != a->hidden || h->map_h_rows != rows) {
+    if (!encode_map(h, &h->map_h, a->hidden, (uint64_t)D, (uint64_t)rows, (uint64_t)D * 2, L::kHalfN)) return FLY_ERR_CUDA;
+    h->map_h_ptr = a->hidden;
+    h->map_h_rows = rows;
+  }
+  const int num_tiles = (V + L::kBlockV - 1) / L::kBlockV;
+  const int grid = num_tiles < h->sm_count ? num_tiles : h->sm_count;
+  for (int64_t row0 = 0; row0 < rows; row0 += L::kMaxPos) {
+    L::Params p;
+    p.R = (int)(rows - row0 < L::kMaxPos ? rows - row0 : L::kMaxPos);
+    const int r16 = (p.R + 15) / 16 * 16;
+    p.n0 = r16 < L::kHalfN ? r16 : L::kHalfN;
+    p.n1 = r16 > L::kHalfN ? r16 - L::kHalfN : 0;
+    p.V = V; p.D = D;
+    p.num_tiles = num_tiles;
+    p.num_kb = (D + L::kBlockK - 1) / L::kBlockK;
+    p.row0 = (int)row0;
+    p.partials = h->lm_partials;
+    p.status = h->lm_status;
+    L::lmhead_verify_kernel<<<grid, L::kThreads, L::kSmemBytes, st>>>(h->map_w, h->map_h, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches++;
+  }
+  const fly::ScanParams sp = scan_params(h, a, h->lm_partials, grid);
+  cudaError_t e = launch_scan(sp, st);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->last_launches++;
+  return FLY_OK;
+}
+
 float theta_to_nats(const fly_verify* h, const fly_verify_args_t* a) {
   double th = a->theta;
   if (a->theta_unit == FLY_THETA_NORMALIZED) th *= std::log((double)h->cfg.vocab);
   return (float)th;
+}
+
+fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, const fly::Partial* partials, int splits) {
+  fly::ScanParams p;
+  p.B = a->B; p.K = a->K; p.V = h->cfg.vocab; p.splits = splits;
+  p.partials = partials;
+  p.tickets = nullptr;
+  p.draft = a->draft;
+  p.theta_nats = theta_to_nats(h, a);
+  p.W = a->W > 64 ? 64 : a->W;
+  p.carry = a->boundary == FLY_BOUNDARY_CARRY;
+  p.state_in = reinterpret_cast<const int32_t*>(a->state_in);
+  p.state_out = reinterpret_cast<int32_t*>(a->state_out);
+  p.accept_len = a->accept_len;
+  p.rollback = a->rollback;
+  p.out_tokens = a->out_tokens;
+  p.target_argmax = a->target_argmax;
+  p.entropy = a->entropy;
+  p.row_flags = a->row_flags;
+  return p;
 }
 
 }  // namespace
@@ -202,7 +293,8 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   if (c->max_batch < 1 || c->max_k < 1 || c->max_k > kMaxK || c->vocab < 1 || c->hidden < 0 || c->device < 0)
     return FLY_ERR_INVALID_ARG;
   if (c->logits_dtype != FLY_F32 && c->logits_dtype != FLY_BF16) return FLY_ERR_INVALID_ARG;
-  if (c->hidden > 0) return FLY_ERR_UNSUPPORTED;  // fused LM-head path: not built yet
+  // the fused path streams both operands with TMA: row pitches must be multiples of 16 bytes
+  if (c->hidden > 0 && (c->hidden % 8 != 0 || c->vocab % 8 != 0)) return FLY_ERR_UNSUPPORTED;
   fly_verify* h = new (std::nothrow) fly_verify();
   if (!h) return FLY_ERR_INVALID_ARG;
   h->cfg = *c;
@@ -218,6 +310,25 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   e = cudaMalloc(&h->tickets, (size_t)c->max_batch * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(h->tickets, 0, (size_t)c->max_batch * sizeof(unsigned int));
   if (e != cudaSuccess) { cudaFree(h->partials); cudaFree(h->tickets); delete h; return FLY_ERR_CUDA; }
+  if (c->hidden > 0) {
+    e = cudaMalloc(&h->lm_partials, (size_t)h->max_rows * h->sm_count * sizeof(fly::Partial));
+    if (e == cudaSuccess) e = cudaMalloc(&h->lm_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(h->lm_status, 0, sizeof(int));
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(fly::lmhead::lmhead_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               fly::lmhead::kSmemBytes);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (e == cudaSuccess) e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || !fn) {
+      fly_status_t st = cuda_fail(h, e);
+      (void)st;
+      cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_partials); cudaFree(h->lm_status);
+      delete h;
+      return FLY_ERR_CUDA;
+    }
+    h->encode_tiled = reinterpret_cast<PFN_cuTensorMapEncodeTiled>(fn);
+  }
   *out = h;
   return FLY_OK;
 }
@@ -228,6 +339,9 @@ fly_status_t fly_verify_destroy(fly_verify_t* h) {
   if (g.ok) {
     cudaFree(h->partials);
     cudaFree(h->tickets);
+    cudaFree(h->lm_partials);
+    cudaFree(h->lm_status);
+    cudaFree(h->st_hidden);
     cudaFree(h->st_logits);
     cudaFree(h->st_ints);
     cudaFree(h->st_entropy);
@@ -255,13 +369,32 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
   return FLY_ERR_INVALID_ARG;
 }
 
+fly_status_t fly_verify_device_status(fly_verify_t* h, void* cuda_stream) {
+  if (!h) return FLY_ERR_INVALID_ARG;
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  int word = 0;
+  if (h->lm_status) {
+    if ((e = cudaMemcpyAsync(&word, h->lm_status, sizeof(int), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+      return cuda_fail(h, e);
+  }
+  if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(h, e);
+  if (word != 0) {
+    if ((e = cudaMemsetAsync(h->lm_status, 0, sizeof(int), st)) != cudaSuccess) return cuda_fail(h, e);
+    return FLY_ERR_TIMEOUT;
+  }
+  return FLY_OK;
+}
+
 int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
 int32_t fly_verify_last_cuda_error(const fly_verify_t* h) { return h ? h->last_cuda_error : 0; }
 
 fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* cuda_stream) {
   fly_status_t s = check_args(h, a);
   if (s != FLY_OK) return s;
-  if (!a->logits) return FLY_ERR_UNSUPPORTED;  // fused LM-head path: not built yet
+  if (!a->logits && h->cfg.hidden <= 0) return FLY_ERR_INVALID_ARG;  // the handle was created without a hidden size
   DeviceGuard g(h->cfg.device);
   if (!g.ok) return FLY_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -269,6 +402,7 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   const int64_t rows = (int64_t)a->B * (a->K + 1);
   const int64_t stride = a->row_stride ? a->row_stride : V;
   h->last_launches = 0;
+  if (!a->logits) return run_fused(h, a, st);
 
   fly::ScanParams p;
   p.B = a->B; p.K = a->K; p.V = V; p.splits = h->last_splits;
@@ -315,7 +449,7 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
 fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, void* cuda_stream) {
   fly_status_t s = check_args(h, a);
   if (s != FLY_OK) return s;
-  if (!a->logits) return FLY_ERR_UNSUPPORTED;
+  if (!a->logits && h->cfg.hidden <= 0) return FLY_ERR_INVALID_ARG;
   DeviceGuard g(h->cfg.device);
   if (!g.ok) return FLY_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -331,7 +465,15 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     if ((e = cudaMalloc(&h->st_ints, ints * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
     if ((e = cudaMalloc(&h->st_entropy, (size_t)(mb * mk1) * sizeof(float))) != cudaSuccess) return cuda_fail(h, e);
   }
-  const size_t logit_bytes = (size_t)(((rows - 1) * stride + V)) * esz;
+  const size_t hidden_bytes = a->logits ? 0 : (size_t)rows * h->cfg.hidden * 2;
+  if (hidden_bytes > h->st_hidden_bytes) {
+    cudaFree(h->st_hidden);
+    h->st_hidden = nullptr;
+    h->st_hidden_bytes = 0;
+    if ((e = cudaMalloc(&h->st_hidden, hidden_bytes)) != cudaSuccess) return cuda_fail(h, e);
+    h->st_hidden_bytes = hidden_bytes;
+  }
+  const size_t logit_bytes = a->logits ? (size_t)(((rows - 1) * stride + V)) * esz : 0;
   if (logit_bytes > h->st_logits_bytes) {
     cudaFree(h->st_logits);
     h->st_logits = nullptr;
@@ -349,7 +491,9 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
   int32_t* d_argmax = d_tokens + mb * mk1;
   int32_t* d_flags = d_argmax + mb * mk1;
 
-  if ((e = cudaMemcpyAsync(h->st_logits, a->logits, logit_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+  if (a->logits && (e = cudaMemcpyAsync(h->st_logits, a->logits, logit_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(h, e);
+  if (!a->logits && (e = cudaMemcpyAsync(h->st_hidden, a->hidden, hidden_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
   if ((e = cudaMemcpyAsync(d_draft, a->draft, (size_t)(B * a->K) * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
@@ -358,7 +502,8 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     return cuda_fail(h, e);
 
   fly_verify_args_t d = *a;
-  d.logits = h->st_logits;
+  d.logits = a->logits ? h->st_logits : nullptr;
+  d.hidden = a->logits ? nullptr : h->st_hidden;  // the weight stays where it is: device memory
   d.draft = d_draft;
   d.state_in = a->state_in ? reinterpret_cast<const fly_state_t*>(d_state_in) : nullptr;
   d.state_out = a->state_out ? reinterpret_cast<fly_state_t*>(d_state_out) : nullptr;

@@ -1,0 +1,426 @@
+// Fused LM-head verification: logits = hidden x weight are formed on the 5th-gen
+// tensor cores (tcgen05.mma, fp32 accumulators in tensor memory) and reduced to
+// the per-row softmax statistics of Eq. 1 / Eq. 5 straight out of tensor memory;
+// the logits never reach global memory.
+//
+// Orientation.  The vocabulary is the MMA's M dimension and the positions are
+// its N dimension ("swap-AB"):  D[v, p] = sum_d weight[d, v] * hidden[p, d].
+//   A = weight tile, 128 vocabulary entries x 64 hidden dims.  weight is [D, V]
+//       with V contiguous, so A is MN-major; TMA lays it down as two boxes of
+//       64 entries (128 bytes) x 64 dims with the 128-byte swizzle.
+//   B = hidden tile, up to 288 positions x 64 hidden dims, K-major, two boxes of
+//       144 positions with the 128-byte swizzle.
+//   D = two accumulators of 128 lanes x 144 fp32 columns (tensor-memory columns
+//       0..143 and 144..287): lane = vocabulary entry, column = position.
+// Up to 288 positions need no padding this way (288 = 2 x 144, both legal MMA
+// N), every weight tile meets all positions while it is in shared memory, and
+// the weights (the only large operand) stream from HBM exactly once.
+//
+// One persistent CTA per SM walks vocabulary tiles blockIdx.x, +gridDim.x, ...
+// Warp roles: 0-3 epilogue (they own the four 32-lane quarters of tensor
+// memory), 4 weight producer, 5 hidden producer, 6 MMA issuer.  Weights and
+// hidden states have rings of their own (deep for the HBM stream, shallow for
+// the L2-resident hidden states).
+//
+// Epilogue.  A thread that reads tensor memory owns one vocabulary entry and
+// sees all positions; the reduction runs over the vocabulary.  The tile is
+// therefore turned through shared memory 32 positions at a time: the four
+// epilogue warps store their 32 x 32 block transposed, then thread
+// (position i, vocabulary quarter q) streams the 32 logits of its quarter and
+// folds them into a running (max, sum 2^t, sum 2^t t, argmax) held in registers
+// for the whole kernel - the same state and the same arithmetic as the row
+// reduction of the logits path, with no cross-lane traffic.  At the end the
+// four quarters are merged and the CTA writes one Partial per position; the
+// acceptance scan folds the gridDim.x partials of every row.
+//
+// Every wait is bounded: a wait that runs out records a code in *status, and
+// all roles fall through to the common exit (tensor memory is released there).
+#pragma once
+#include <cuda.h>
+
+#include "fly_common.cuh"
+
+namespace fly {
+namespace lmhead {
+
+constexpr int kBlockV = 128;   // vocabulary entries per tile (MMA M)
+constexpr int kBlockK = 64;    // hidden dims per stage: one 128-byte swizzle row of bf16
+constexpr int kMmaK = 16;      // hidden dims per tcgen05.mma (bf16)
+constexpr int kHalfN = 144;    // positions per accumulator (MMA N <= 256, multiple of 16)
+constexpr int kMaxPos = 2 * kHalfN;
+constexpr int kStagesW = 6;    // weight ring
+constexpr int kStagesH = 3;    // hidden ring
+constexpr int kBytesW = kBlockK * kBlockV * 2;      // 16 KB per stage
+constexpr int kBytesWBox = kBlockK * 64 * 2;        // one TMA box: 64 entries x 64 dims
+constexpr int kBytesHHalf = kHalfN * kBlockK * 2;   // 18 KB
+constexpr int kBytesH = 2 * kBytesHHalf;
+constexpr int kChunk = 32;                          // positions turned through shared memory at a time
+constexpr int kChunks = kMaxPos / kChunk;           // 9
+constexpr int kTurnRow = kBlockV + 4;               // words per position row (+4: conflict-free 128-bit reads)
+constexpr int kTurnBytes = kChunk * kTurnRow * 4;
+constexpr int kEpiThreads = 128;
+constexpr int kThreads = 224;
+constexpr int kTmemCols = 512;
+
+constexpr int kOffW = 0;
+constexpr int kOffH = kOffW + kStagesW * kBytesW;
+constexpr int kOffTurn = kOffH + kStagesH * kBytesH;
+constexpr int kOffBar = kOffTurn + kTurnBytes;
+constexpr int kNumBars = 2 * kStagesW + 2 * kStagesH + 2;
+constexpr int kOffMisc = kOffBar + kNumBars * 8;
+constexpr int kSmemBytes = kOffMisc + 32 + 1024;    // + slack to align the base to 1024 bytes
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
+static_assert(kMaxPos * 4 * 16 <= kStagesW * kBytesW, "final merge buffer reuses the weight ring");
+
+constexpr int kErrTimeoutProducer = 1, kErrTimeoutMma = 2, kErrTimeoutEpilogue = 3;
+constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;  // far above any legitimate wait (a tile takes ~50 us)
+
+struct Params {
+  int R;          // positions handled by this launch (1..288)
+  int n0, n1;     // MMA N of the two accumulators (multiples of 16; n1 may be 0)
+  int V, D;
+  int num_tiles;  // ceil(V / 128)
+  int num_kb;     // ceil(D / 64)
+  int row0;       // first row of this launch in hidden / partials
+  Partial* partials;  // [rows, gridDim.x]
+  int* status;        // 0, or the code of the first wait that ran out
+};
+
+// ---- small PTX wrappers ------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase of `bar` with the given parity to complete.  Gives up when
+// the limit passes or when another role has already reported a failure.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63) == 0) {
+      if (*(volatile int*)status != 0) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem], one CTA, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// ---- descriptors ---------------------------------------------------------------
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading and
+// stride byte offsets in 16-byte units, descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, A MN-major (vocabulary
+// contiguous), B K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(kBlockV >> 4) << 24);
+}
+
+// Running statistics of one (position, vocabulary quarter) stream.
+struct Stream {
+  float mx, S, u;
+  int idx;
+};
+
+// Folds 32 consecutive vocabulary entries x[0..31] (the first one has index v0) into st.
+__device__ __forceinline__ void fold32(Stream& st, float (&x)[32], int v0) {
+  float lm = kMaskFloor;
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    x[e] = max_nan_f32(x[e], kMaskFloor);  // masked entries stay finite; NaN survives and ends in S
+    lm = fmaxf(lm, x[e]);
+  }
+  if (lm > st.mx) {  // the maximum moves: rebase the sums and record the first entry that holds it
+    const float d = (st.mx - lm) * kLog2e;
+    const float sc = ex2_approx(d);
+    st.u = sc * fmaf(d, st.S, st.u);
+    st.S *= sc;
+    st.mx = lm;
+    int first = 31;
+#pragma unroll
+    for (int e = 31; e >= 0; --e)
+      if (x[e] == lm) first = e;
+    st.idx = v0 + first;
+  }
+  const float nr = -st.mx * kLog2e;
+  float S0 = 0.f, S1 = 0.f, u0 = 0.f, u1 = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; e += 2) {
+    const float t0 = fmaf(x[e], kLog2e, nr), t1 = fmaf(x[e + 1], kLog2e, nr);
+    const float e0 = ex2_approx(t0), e1 = ex2_approx(t1);
+    S0 += e0;
+    u0 = fmaf(e0, t0, u0);
+    S1 += e1;
+    u1 = fmaf(e1, t1, u1);
+  }
+  st.S += S0 + S1;
+  st.u += u0 + u1;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_h,
+                     const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
+  uint8_t* gbase = smem_raw + (base - raw);
+  const uint32_t bar0 = base + kOffBar;
+  auto full_w = [&](int s) { return bar0 + 8u * s; };
+  auto empty_w = [&](int s) { return bar0 + 8u * (kStagesW + s); };
+  auto full_h = [&](int s) { return bar0 + 8u * (2 * kStagesW + s); };
+  auto empty_h = [&](int s) { return bar0 + 8u * (2 * kStagesW + kStagesH + s); };
+  const uint32_t tmem_full = bar0 + 8u * (2 * kStagesW + 2 * kStagesH);
+  const uint32_t tmem_empty = tmem_full + 8u;
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1] epilogue go flag
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStagesW; ++s) { mbar_init(full_w(s), 1); mbar_init(empty_w(s), 1); }
+    for (int s = 0; s < kStagesH; ++s) { mbar_init(full_h(s), 1); mbar_init(empty_h(s), 1); }
+    mbar_init(tmem_full, 1);
+    mbar_init(tmem_empty, kEpiThreads);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {  // one warp allocates all of tensor memory (one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffMisc),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+
+  const int my_tiles = blockIdx.x < p.num_tiles ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+
+  if (warp == 4) {
+    // ---------------- weight producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        const int v0 = ((int)blockIdx.x + t * (int)gridDim.x) * kBlockV;
+        for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
+          const int s = issued % kStagesW;
+          const uint32_t ph = (issued / kStagesW) & 1;
+          if (!mbar_wait(empty_w(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
+          mbar_expect_tx(full_w(s), kBytesW);
+          const uint32_t dst = base + kOffW + s * kBytesW;
+          tma_load_2d(dst, &map_w, v0, kb * kBlockK, full_w(s));
+          tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, full_w(s));
+        }
+      }
+      // copies still in flight must land before the CTA gives its shared memory back
+      for (int i = issued > kStagesW ? issued - kStagesW : 0; i < issued; ++i)
+        mbar_wait(full_w(i % kStagesW), (i / kStagesW) & 1, p.status, kErrTimeoutProducer);
+    }
+  } else if (warp == 5) {
+    // ---------------- hidden-state producer ----------------
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      const uint32_t bytes = p.n1 > 0 ? kBytesH : kBytesHHalf;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
+          const int s = issued % kStagesH;
+          const uint32_t ph = (issued / kStagesH) & 1;
+          if (!mbar_wait(empty_h(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
+          mbar_expect_tx(full_h(s), bytes);
+          const uint32_t dst = base + kOffH + s * kBytesH;
+          tma_load_2d(dst, &map_h, kb * kBlockK, p.row0, full_h(s));
+          if (p.n1 > 0) tma_load_2d(dst + kBytesHHalf, &map_h, kb * kBlockK, p.row0 + kHalfN, full_h(s));
+        }
+      }
+      for (int i = issued > kStagesH ? issued - kStagesH : 0; i < issued; ++i)
+        mbar_wait(full_h(i % kStagesH), (i / kStagesH) & 1, p.status, kErrTimeoutProducer);
+    }
+  } else if (warp == 6) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc0 = instr_desc(p.n0), idesc1 = instr_desc(p.n1 > 0 ? p.n1 : 16);
+      int it = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        // the epilogue must have drained the accumulators of the previous tile
+        if (!mbar_wait(tmem_empty, (t & 1) ^ 1, p.status, kErrTimeoutMma)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+          const int sw = it % kStagesW, sh = it % kStagesH;
+          if (!mbar_wait(full_w(sw), (it / kStagesW) & 1, p.status, kErrTimeoutMma) ||
+              !mbar_wait(full_h(sh), (it / kStagesH) & 1, p.status, kErrTimeoutMma)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t aw = base + kOffW + sw * kBytesW;
+          const uint32_t bh = base + kOffH + sh * kBytesH;
+#pragma unroll
+          for (int ks = 0; ks < kBlockK / kMmaK; ++ks) {
+            // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden
+            // dims 1024 bytes apart (stride offset); 16 hidden dims further = 16 rows of 128 bytes.
+            const uint64_t da = smem_desc(aw + ks * (kMmaK * 128), kBytesWBox, 1024);
+            // B, K-major: groups of 8 positions 1024 bytes apart; 16 hidden dims further = 32 bytes.
+            const uint64_t db0 = smem_desc(bh + ks * (kMmaK * 2), 16, 1024);
+            const uint32_t acc = (kb | ks) != 0;
+            mma_bf16(tmem, da, db0, idesc0, acc);
+            if (p.n1 > 0) {
+              const uint64_t db1 = smem_desc(bh + kBytesHHalf + ks * (kMmaK * 2), 16, 1024);
+              mma_bf16(tmem + kHalfN, da, db1, idesc1, acc);
+            }
+          }
+          mma_commit(empty_w(sw));  // the stage may be refilled once these MMAs have read it
+          mma_commit(empty_h(sh));
+        }
+        if (ok) mma_commit(tmem_full);
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 0..3, thread = (position lane, vocabulary quarter warp) ----------------
+    Stream st[kChunks];
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) { st[c].mx = kMaskFloor; st[c].S = 0.f; st[c].u = 0.f; st[c].idx = kIdxNone; }
+    float* turn = reinterpret_cast<float*>(gbase + kOffTurn);
+    const int nchunks = (p.R + kChunk - 1) / kChunk;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    for (int t = 0; t < my_tiles; ++t) {
+      const int tile = (int)blockIdx.x + t * (int)gridDim.x;
+      if (threadIdx.x == 0) misc[1] = mbar_wait(tmem_full, t & 1, p.status, kErrTimeoutEpilogue) ? 1u : 0u;
+      epi_bar();
+      const bool go = misc[1] != 0;  // one thread waits, all take the same decision
+      if (!go) break;
+      tc_fence_after();
+      const int v0 = tile * kBlockV + warp * 32;
+      const int limit = p.V - v0;  // entries of this quarter that exist
+#pragma unroll
+      for (int c = 0; c < kChunks; ++c) {
+        if (c < nchunks) {
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_base + (uint32_t)(c * kChunk), r);
+          if (c == nchunks - 1) {  // last read of this tile: hand the accumulators back to the MMA issuer
+            tc_fence_before();
+            mbar_arrive(tmem_empty);
+          }
+          epi_bar();  // everyone is done reading the previous block
+#pragma unroll
+          for (int i = 0; i < 32; ++i) turn[i * kTurnRow + warp * 32 + lane] = __uint_as_float(r[i]);
+          epi_bar();
+          float x[32];
+          const float4* src = reinterpret_cast<const float4*>(turn + lane * kTurnRow + warp * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float4 q = src[j];
+            x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
+          }
+          if (limit < 32) {  // ragged vocabulary: entries past V do not exist
+#pragma unroll
+            for (int e = 0; e < 32; ++e)
+              if (e >= limit) x[e] = kMaskFloor;
+          }
+          fold32(st[c], x, v0);
+        }
+      }
+    }
+    // Merge the four vocabulary quarters of every position and write the CTA's partial state.
+    // The weight ring is free by now: every MMA that read it has completed (tmem_full of the last tile).
+    epi_bar();
+    Partial* buf = reinterpret_cast<Partial*>(gbase + kOffW);
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      Partial q;
+      q.mx = st[c].mx; q.S = st[c].S; q.u = st[c].u; q.idx = st[c].idx;
+      buf[(c * kChunk + lane) * 4 + warp] = q;
+    }
+    epi_bar();
+    for (int pos = threadIdx.x; pos < p.R; pos += kEpiThreads) {
+      Partial a = buf[pos * 4];
+      merge_partial(a, buf[pos * 4 + 1]);
+      merge_partial(a, buf[pos * 4 + 2]);
+      merge_partial(a, buf[pos * 4 + 3]);
+      p.partials[(int64_t)(p.row0 + pos) * gridDim.x + blockIdx.x] = a;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+}  // namespace lmhead
+}  // namespace fly

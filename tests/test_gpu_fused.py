@@ -1,0 +1,124 @@
+"""Parity of the fused LM-head path (tcgen05 GEMM with the entropy / argmax
+epilogue, called through the C ABI) with the fp64 oracle: the oracle forms the
+logits as the exact fp64 product of the bf16 inputs and verifies them as usual."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fly_oracle as O
+from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, binding as Bd, synthetic as S, verify_fused
+from tests._parity import assert_parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def fused_case(B, K, D, V, step=0, weight_std=None, theta=1.0, min_gap=1e-3, guard=1e-3):
+    """hidden, weight (bf16, device), draft and the oracle's logits for one step.  A hidden row is redrawn
+    while its two largest fp64 logits are closer than min_gap (fp32 accumulation could then pick the other
+    one) or its entropy is within `guard` of theta."""
+    w = S.shrink(S.FUSED, B=B, K=K, V=V, hidden=D, weight_std=weight_std or 2.0 / np.sqrt(D))
+    weight = S.make_weight(w, device="cpu")
+    hidden = S.make_hidden(w, step, device="cpu")
+    wd = weight.double().numpy()
+    for attempt in range(1, 8):
+        logits = O.lm_head_logits(hidden.double().numpy(), wd)
+        top2 = np.partition(logits, V - 2, axis=1)[:, V - 2:]
+        H = O.row_stats(logits)[0]
+        bad = np.nonzero((np.abs(top2[:, 1] - top2[:, 0]) < min_gap) | (np.abs(H - theta) < guard))[0]
+        if bad.size == 0:
+            break
+        fresh = S.make_hidden(w, step, device="cpu", attempt=attempt)
+        hidden[torch.as_tensor(bad)] = fresh[torch.as_tensor(bad)]
+    else:
+        raise RuntimeError("could not separate the top two logits of every row")
+    y = torch.as_tensor(logits.argmax(axis=1)).view(-1, 1)
+    draft = S.make_draft(w, step, y)
+    return w, hidden.to(DEV), weight.to(DEV), draft.to(DEV), logits
+
+
+def run_and_check(B, K, D, V, theta=1.0, W=3, boundary="reject", state=None, **kw):
+    w, hidden, weight, draft, logits = fused_case(B, K, D, V, theta=theta, **kw)
+    fv = FlyVerify(B, K, V, "bf16", hidden=D)
+    out = VerifyBuffers(B, K, DEV)
+    if state is not None:
+        out.state.copy_(torch.as_tensor(state, dtype=torch.int32))
+    verify_fused(fv, hidden, weight, draft, out, theta=theta, W=W, boundary=boundary,
+                 stream=torch.cuda.current_stream().cuda_stream)
+    assert fv.device_status(torch.cuda.current_stream().cuda_stream) == Bd.FLY_OK
+    ref = O.verify_batch(logits.reshape(B, K + 1, V), draft.cpu().numpy(), theta, W, boundary=boundary,
+                         state_in=None if state is None else np.asarray(state))
+    err = assert_parity(out, ref, f"fused B={B} K={K} D={D} V={V}")
+    fv.close()
+    return err, out, ref
+
+
+@pytest.mark.parametrize("B,K", [(1, 1), (2, 7), (4, 8), (16, 8), (17, 8), (32, 8)])
+def test_position_counts_up_to_one_block(B, K):
+    # 2 .. 288 positions: one accumulator, both, a ragged second one
+    run_and_check(B, K, D=256, V=1024)
+
+
+@pytest.mark.parametrize("D,V", [(64, 128), (128, 256), (512, 4096), (200, 1000), (1024, 19000)])
+def test_hidden_and_vocabulary_sizes(D, V):
+    # one k-block, several, a ragged last k-block (200), a ragged last vocabulary tile (1000, 19000),
+    # more tiles than SMs (19000 -> 149 tiles)
+    run_and_check(4, 8, D=D, V=V)
+
+
+def test_more_positions_than_one_block_and_carry_state():
+    # 360 positions: two launches over the weight; carried state in and out
+    B, K = 40, 8
+    state = [[(b % 3), 4, 11] for b in range(B)]
+    run_and_check(B, K, D=256, V=2048, boundary="carry", state=state)
+
+
+def test_theta_and_window_settings():
+    for theta, W in [(0.5, 1), (2.0, 5), (float("inf"), 3), (0.0, 0)]:
+        run_and_check(8, 8, D=256, V=2048, theta=theta, W=W)
+
+
+def test_fused_matches_logits_path_on_materialised_logits():
+    # same step through both paths: integers must agree, entropy within tolerance (the logits path reads the
+    # product rounded to bf16, so only a loose entropy bound holds there; integers are compared where the
+    # rounded logits keep the same argmax)
+    B, K, D, V = 8, 8, 512, 8192
+    w, hidden, weight, draft, logits = fused_case(B, K, D, V, step=3)
+    fv = FlyVerify(B, K, V, "f32", hidden=D)
+    out_f = VerifyBuffers(B, K, DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    verify_fused(fv, hidden, weight, draft, out_f, stream=st)
+    lg = torch.as_tensor(logits, dtype=torch.float32).view(B, K + 1, V).to(DEV)
+    out_l = VerifyBuffers(B, K, DEV)
+    from paper_2511_22972_b200 import verify
+    verify(fv, lg, draft, out_l, stream=st)
+    torch.cuda.synchronize()
+    assert torch.equal(out_f.target_argmax, out_l.target_argmax)
+    assert torch.equal(out_f.accept_len, out_l.accept_len)
+    assert torch.equal(out_f.out_tokens, out_l.out_tokens)
+    assert (out_f.entropy - out_l.entropy).abs().max().item() <= 1e-4
+
+
+def test_host_buffer_entry_point_on_the_fused_path():
+    B, K, D, V = 4, 8, 256, 2048
+    w, hidden, weight, draft, logits = fused_case(B, K, D, V, step=5)
+    fv = FlyVerify(B, K, V, "bf16", hidden=D)
+    out = VerifyBuffers(B, K, "cpu", pinned=True)
+    verify_fused(fv, hidden.cpu().pin_memory(), weight, draft.cpu().pin_memory(), out, host=True,
+                 stream=torch.cuda.current_stream().cuda_stream)
+    ref = O.verify_batch(logits.reshape(B, K + 1, V), draft.cpu().numpy(), 1.0, 3)
+    assert_parity(out, ref, "fused host")
+
+
+def test_fused_misuse():
+    fv = FlyVerify(2, 4, 1024, "bf16")                       # no hidden size: the fused path is not available
+    out = VerifyBuffers(2, 4, DEV)
+    hidden = torch.zeros(10, 64, dtype=torch.bfloat16, device=DEV)
+    weight = torch.zeros(64, 1024, dtype=torch.bfloat16, device=DEV)
+    draft = torch.zeros(2, 4, dtype=torch.int32, device=DEV)
+    with pytest.raises(Bd.FlyError) as e:
+        verify_fused(fv, hidden, weight, draft, out)
+    assert e.value.status == Bd.FLY_ERR_INVALID_ARG
+    with pytest.raises(Bd.FlyError) as e:
+        FlyVerify(2, 4, 1001, "bf16", hidden=64)             # row pitch of the weight not a multiple of 16 bytes
+    assert e.value.status == Bd.FLY_ERR_UNSUPPORTED
