@@ -189,6 +189,153 @@ def oracle_rate(w, seconds_budget=12.0):
     return rows_done / t_used, f"{steps} steps of {ws.B} sequences x {ws.K + 1} rows x V={ws.V} ({w.dtype} widened to fp64)", 1
 
 
+def measured_tensor_peak():
+    """(burst, sustained) bf16 TFLOP/s of this machine's B200s, and where the numbers come from."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1590.0, 1400.0, "fallback"
+
+
+def fused_oracle_sample(w, weight_cpu, seq, step):
+    """The oracle on `seq` sequences of the fused workload (all V): exact fp64 logits, then the usual
+    verification.  The product is taken in vocabulary slices so that the fp64 copy of the weight never
+    exists as a whole; only the oracle calls are timed.  Returns (seconds, rows)."""
+    import numpy as np
+    from oracle import fly_oracle as O
+    from paper_2511_22972_b200 import synthetic as S
+    ws = S.shrink(w, B=seq)
+    hidden = S.make_hidden(ws, step, device="cpu").double().numpy()
+    draft = np.random.default_rng(step).integers(0, w.V, size=(seq, w.K)).astype(np.int32)
+    t, parts = 0.0, []
+    for v0 in range(0, w.V, 16032):
+        wd = weight_cpu[:, v0:v0 + 16032].double().numpy()
+        t0 = time.perf_counter()
+        parts.append(O.lm_head_logits(hidden, wd))
+        t += time.perf_counter() - t0
+    t0 = time.perf_counter()
+    logits = np.concatenate(parts, axis=1).reshape(seq, w.K + 1, w.V)
+    O.verify_batch(logits, draft, w.theta, w.W, boundary=w.boundary)
+    t += time.perf_counter() - t0
+    return t, ws.rows
+
+
+def run_fused(args, w):
+    """The fused LM-head workload: hidden [B*(K+1), D] x weight [D, V] with the verification in the epilogue."""
+    import torch
+    from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, binding as Bd, dist as D, synthetic as S
+    args.steps = args.steps or 200
+    args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
+    ranks = D.init_from_env("nccl")
+    assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
+    torch.cuda.set_device(ranks.local_rank)
+    device = torch.device("cuda", ranks.local_rank)
+    weight = S.make_weight(w, device=device)
+    nbuf = 4
+    hiddens = [S.make_hidden(w, i, device=device) for i in range(nbuf)]
+    # synthetic drafter: the (library, fp32) argmax with p = 0.7, else uniform over V
+    drafts = [S.make_draft(w, i, (h.float() @ weight.float()).argmax(dim=1, keepdim=True)) for i, h in enumerate(hiddens)]
+    torch.cuda.synchronize()
+    out = VerifyBuffers(w.B, w.K, device)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16", device=ranks.local_rank, hidden=w.hidden)
+    mk = lambda h, d, o: fv.make_args(w.B, w.K, d, o.accept_len, o.out_tokens, hidden=h, weight=weight, theta=w.theta,
+                                      W=w.W, boundary=w.boundary, state_out=o.state, rollback=o.rollback,
+                                      target_argmax=o.target_argmax, entropy=o.entropy, row_flags=o.row_flags)
+    arglist = [mk(h, d, out) for h, d in zip(hiddens, drafts)]
+    stream = torch.cuda.Stream(device=device)
+    with ClockSampler(ranks.local_rank) as clk:
+        ms_total = time_steps(fv, arglist, stream, args.steps, args.warmup, ranks, "stream")
+        launches_per_step = fv.last_launch_count
+    if fv.device_status(stream.cuda_stream) != Bd.FLY_OK:
+        raise SystemExit("a bounded device-side wait ran out: the measurement is void")
+    ms_per_step = ms_total / args.steps
+    rows_all = w.rows * ranks.world
+    value = rows_all / (ms_per_step * 1e-3)
+
+    # end to end: hidden states and drafts come from pinned host memory every step, results go back
+    e2e_steps = max(10, min(100, args.steps // 2))
+    hout = VerifyBuffers(w.B, w.K, device, pinned=True)
+    hargs = [mk(h.cpu().pin_memory(), d.cpu().pin_memory(), hout) for h, d in zip(hiddens[:2], drafts[:2])]
+    keep = [a for a in hargs]
+    raw = stream.cuda_stream
+    for i in range(3):
+        fv.run_host(hargs[i % 2], raw)
+    D.barrier(ranks)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        fv.run_host(hargs[i % 2], raw)
+    torch.cuda.synchronize()
+    e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
+    h2d = w.rows * w.hidden * 2 + w.B * w.K * 4
+    d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
+
+    flops = 2.0 * w.rows * w.hidden * w.V
+    burst, sustained, kind = measured_tensor_peak()
+    achieved = flops / (ms_per_step * 1e-3) / 1e12
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "hidden": w.hidden,
+                   "theta_nats": w.theta, "W": w.W, "boundary": w.boundary, "parallelism": f"dp{ranks.world}",
+                   "launch": "stream", "l2": f"the weight ({w.hidden * w.V * 2 / 1e9:.2f} GB, read once per step) is larger than L2"},
+        "tflops": achieved,
+        "roofline": {"bound": "tensor", "kernel": "lmhead_verify_kernel (tcgen05 GEMM + entropy/argmax epilogue)",
+                     "achieved": achieved, "peak": burst, "peak_kind": f"of {kind} (bf16 burst)", "unit": "TFLOP/s",
+                     "frac": achieved / burst, "frac_of_sustained": achieved / sustained, "flops_per_launch": flops,
+                     "us_per_launch": ms_per_step * 1e3,
+                     "note": "duration = whole step (GEMM kernel + acceptance-scan kernel, the latter ~3 us)",
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "hbm_gbs": (w.hidden * w.V * 2 + w.rows * w.hidden * 2) / (ms_per_step * 1e-3) / 1e9,
+        "e2e": {"value": rows_all * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                "api": "fly_verify_run_host (hidden states and drafts in pinned host buffers; weight resident)"},
+        "gpu_launches": launches_per_step * args.steps,
+        "clocks": clk.summary(),
+    }
+    if ranks.is_main and ranks.world == 1 and not args.no_cpu_baseline:
+        wc = weight.cpu()
+        t, rows = fused_oracle_sample(w, wc, 1, 0)
+        line["cpu_baseline"] = {"value": rows / t, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
+                                "sample": f"1 of {w.B} sequences ({rows} rows, all V={w.V}): fp64 matmul (BLAS threads) + verification (1 thread)"}
+    if ranks.is_main:
+        print(json.dumps(line), flush=True)
+    fv.close()
+    D.finalize(ranks)
+
+
+def run_reference_fused(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2511_22972_b200 import synthetic as S
+    weight = S.make_weight(w, device="cpu")
+    for i in range(args.warmup):
+        fused_oracle_sample(w, weight, 1, i)
+    tot, rows = 0.0, 0
+    for i in range(args.steps):
+        t, r = fused_oracle_sample(w, weight, 1, 100 + i)
+        tot += t
+        rows += r
+    value = rows / tot
+    sample = f"each step = 1 of {w.B} sequences ({w.K + 1} rows, all V={w.V}), fp64 matmul + verification"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "K": w.K, "V": w.V, "hidden": w.hidden, "theta_nats": w.theta,
+                   "W": w.W, "boundary": w.boundary, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def run_reference(args, w):
     """--impl reference: the oracle on the host cores; rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
@@ -241,16 +388,22 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="plain stream order between steps (no programmatic dependent launch)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--vocab", type=int, default=None, help="run the workload's recipe at another vocabulary size "
+                    "(smaller cases for profiler captures); recorded in config")
+    ap.add_argument("--batch", type=int, default=None, help="run the workload's recipe at another batch size")
     args = ap.parse_args()
 
     from paper_2511_22972_b200 import synthetic as S
     w = S.WORKLOADS[args.workload]
-    if w.hidden:
-        raise SystemExit("the fused LM-head workload is not built yet")
+    if args.vocab or args.batch:
+        w = S.shrink(w, V=args.vocab or w.V, B=args.batch or w.B)
     if args.impl == "reference":
         args.steps = args.steps or 5
         args.warmup = 1 if args.warmup is None else args.warmup
-        run_reference(args, w)
+        (run_reference_fused if w.hidden else run_reference)(args, w)
+        return
+    if w.hidden:
+        run_fused(args, w)
         return
     args.steps = args.steps or 20000
     args.warmup = 20 if args.warmup is None else max(args.warmup, 3)

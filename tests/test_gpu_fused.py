@@ -122,3 +122,51 @@ def test_fused_misuse():
     with pytest.raises(Bd.FlyError) as e:
         FlyVerify(2, 4, 1001, "bf16", hidden=64)             # row pitch of the weight not a multiple of 16 bytes
     assert e.value.status == Bd.FLY_ERR_UNSUPPORTED
+
+
+def test_full_size_head_on_sampled_sequences():
+    """The Llama-3.1-70B head shape of the benchmark (288 positions x 8192 x 128256), in the launch
+    configuration the benchmark times.  The oracle cannot form all 288 x 128256 fp64 logits in seconds, so
+    two whole sequences (18 rows) are verified exactly and the rest is checked through properties."""
+    w = S.FUSED
+    B, K, V, D = w.B, w.K, w.V, w.hidden
+    weight = S.make_weight(w, device=DEV)
+    hidden = S.make_hidden(w, 0, device=DEV)
+    sample = [3, 20]
+    hs = hidden.view(B, K + 1, D)[sample].reshape(-1, D).double().cpu().numpy()
+    wc = weight.cpu()
+    parts = [O.lm_head_logits(hs, wc[:, v0:v0 + 16032].double().numpy()) for v0 in range(0, V, 16032)]
+    logits = np.concatenate(parts, axis=1)                       # [18, V] fp64
+    top2 = np.partition(logits, V - 2, axis=1)[:, V - 2:]
+    assert (top2[:, 1] - top2[:, 0]).min() >= 1e-3, "redraw: two logits of a sampled row are too close"
+    y = logits.argmax(axis=1).reshape(len(sample), K + 1)
+    g = torch.Generator().manual_seed(7)
+    draft = torch.randint(0, V, (B, K), generator=g, dtype=torch.int32)
+    for n, b in enumerate(sample):                               # the oracle's token with p = 0.7, else uniform
+        keep = torch.rand(K, generator=g) < 0.7
+        draft[b, keep] = torch.as_tensor(y[n, :K], dtype=torch.int32)[keep]
+    draft = draft.to(DEV)
+    fv = FlyVerify(B, K, V, "bf16", hidden=D)
+    out = VerifyBuffers(B, K, DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    verify_fused(fv, hidden, weight, draft, out, theta=w.theta, W=w.W, stream=st)
+    assert fv.device_status(st) == Bd.FLY_OK
+    assert fv.last_launch_count == 2
+    ref = O.verify_batch(logits.reshape(len(sample), K + 1, V), draft[sample].cpu().numpy(), w.theta, w.W)
+    assert np.array_equal(out.target_argmax[sample].cpu().numpy(), ref.target_argmax)
+    assert np.abs(out.entropy[sample].double().cpu().numpy() - ref.entropy).max() <= 1e-4
+    assert np.array_equal(out.accept_len[sample].cpu().numpy(), ref.accept_len)
+    assert np.array_equal(out.out_tokens[sample].cpu().numpy(), ref.out_tokens)
+    # every sequence: properties that hold whatever the logits are
+    s = out.accept_len.cpu().numpy()
+    toks = out.out_tokens.cpu().numpy()
+    am = out.target_argmax.cpu().numpy()
+    dr = draft.cpu().numpy()
+    H = out.entropy.cpu().numpy()
+    assert ((s >= 1) & (s <= K + 1)).all() and (out.row_flags == 0).all()
+    assert ((H > 0) & (H <= np.log(V) + 1e-4)).all() and ((am >= 0) & (am < V)).all()
+    for b in range(B):
+        assert (toks[b, :s[b] - 1] == dr[b, :s[b] - 1]).all() and toks[b, s[b] - 1] == am[b, s[b] - 1]
+        assert (toks[b, s[b]:] == -1).all()
+        first_mismatch = next((i + 1 for i in range(K) if dr[b, i] != am[b, i]), K + 1)
+        assert s[b] >= first_mismatch                              # s_FLy >= s_standard (Eq. 3 vs Eq. 11)
