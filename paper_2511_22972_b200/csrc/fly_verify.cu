@@ -52,6 +52,7 @@ struct fly_verify {
   // fused LM-head path (cfg.hidden > 0)
   fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]
   int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
+  int lm_pairs = 0;                     // CTA pairs that can be resident at once
   PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
   CUtensorMap map_w, map_h;             // cached for (map_w_ptr, map_h_ptr, map_h_rows)
   const void* map_w_ptr = nullptr;
@@ -214,12 +215,12 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     h->map_w_ptr = a->weight;
   }
   if (h->map_h_ptr != a->hidden || h->map_h_rows != rows) {
-    if (!encode_map(h, &h->map_h, a->hidden, (uint64_t)D, (uint64_t)rows, (uint64_t)D * 2, L::kHalfN)) return FLY_ERR_CUDA;
+    if (!encode_map(h, &h->map_h, a->hidden, (uint64_t)D, (uint64_t)rows, (uint64_t)D * 2, L::kBoxPos)) return FLY_ERR_CUDA;
     h->map_h_ptr = a->hidden;
     h->map_h_rows = rows;
   }
-  const int num_tiles = (V + L::kBlockV - 1) / L::kBlockV;
-  const int grid = num_tiles < h->sm_count ? num_tiles : h->sm_count;
+  const int num_tiles = (V + L::kPairV - 1) / L::kPairV;  // one tile = 256 vocabulary entries = one CTA pair
+  const int grid = 2 * (num_tiles < h->lm_pairs ? num_tiles : h->lm_pairs);
   for (int64_t row0 = 0; row0 < rows; row0 += L::kMaxPos) {
     L::Params p;
     p.R = (int)(rows - row0 < L::kMaxPos ? rows - row0 : L::kMaxPos);
@@ -317,6 +318,26 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(fly::lmhead::lmhead_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                fly::lmhead::kSmemBytes);
+    if (e == cudaSuccess) {
+      // how many pairs (clusters of two CTAs, one CTA per SM) fit on the device at once
+      cudaLaunchConfig_t lc;
+      memset(&lc, 0, sizeof(lc));
+      lc.gridDim = dim3((unsigned)(h->sm_count & ~1));
+      lc.blockDim = dim3(fly::lmhead::kThreads);
+      lc.dynamicSmemBytes = fly::lmhead::kSmemBytes;
+      cudaLaunchAttribute at[1];
+      at[0].id = cudaLaunchAttributeClusterDimension;
+      at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+      lc.attrs = at;
+      lc.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, fly::lmhead::lmhead_verify_kernel, &lc) != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = h->sm_count / 2;
+      }
+      h->lm_pairs = n < h->sm_count / 2 ? n : h->sm_count / 2;
+      if (h->lm_pairs < 1) h->lm_pairs = 1;
+    }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (e == cudaSuccess) e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);

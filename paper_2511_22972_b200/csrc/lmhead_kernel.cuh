@@ -5,22 +5,28 @@
 //
 // Orientation.  The vocabulary is the MMA's M dimension and the positions are
 // its N dimension ("swap-AB"):  D[v, p] = sum_d weight[d, v] * hidden[p, d].
-//   A = weight tile, 128 vocabulary entries x 64 hidden dims.  weight is [D, V]
-//       with V contiguous, so A is MN-major; TMA lays it down as two boxes of
-//       64 entries (128 bytes) x 64 dims with the 128-byte swizzle.
-//   B = hidden tile, up to 288 positions x 64 hidden dims, K-major, two boxes of
-//       144 positions with the 128-byte swizzle.
-//   D = two accumulators of 128 lanes x 144 fp32 columns (tensor-memory columns
-//       0..143 and 144..287): lane = vocabulary entry, column = position.
-// Up to 288 positions need no padding this way (288 = 2 x 144, both legal MMA
-// N), every weight tile meets all positions while it is in shared memory, and
-// the weights (the only large operand) stream from HBM exactly once.
+// Two CTAs on neighbouring SMs work as one pair (tcgen05 cta_group::2) on a tile
+// of 256 vocabulary entries x up to 288 positions:
+//   A = weight tile.  Each CTA holds ITS 128 vocabulary entries x 64 hidden dims.
+//       weight is [D, V] with V contiguous, so A is MN-major; TMA lays it down as
+//       two boxes of 64 entries (128 bytes) x 64 dims with the 128-byte swizzle.
+//   B = hidden tile, K-major, 128-byte swizzle.  The pair shares it: each CTA
+//       loads HALF of the positions of each accumulator (2 x 72 rows), the MMA
+//       reads both halves.  This halves the hidden-state traffic per SM, which is
+//       what bounds a one-CTA version of this kernel (the hidden tile is
+//       re-fetched from L2 for every vocabulary tile).
+//   D = two accumulators of 144 fp32 columns (tensor-memory columns 0..143 and
+//       144..287) in each CTA: lane = one of the CTA's 128 vocabulary entries,
+//       column = position.
+// Up to 288 positions need no padding this way (288 = 2 x 144, a legal MMA N),
+// every weight tile meets all positions while it is in shared memory, and the
+// weights (the only large operand) stream from HBM exactly once.
 //
-// One persistent CTA per SM walks vocabulary tiles blockIdx.x, +gridDim.x, ...
-// Warp roles: 0-3 epilogue (they own the four 32-lane quarters of tensor
-// memory), 4 weight producer, 5 hidden producer, 6 MMA issuer.  Weights and
-// hidden states have rings of their own (deep for the HBM stream, shallow for
-// the L2-resident hidden states).
+// Pairs are persistent: pair i walks vocabulary tiles i, i + #pairs, ...  Warp
+// roles in each CTA: 0-3 epilogue (they own the four 32-lane quarters of tensor
+// memory), 4 weight producer, 5 hidden producer, 6 MMA issuer (leader CTA only).
+// "Full" barriers live in the leader: both CTAs' TMA loads report their bytes
+// there.  The leader's tcgen05.commit releases a stage in both CTAs.
 //
 // Epilogue.  A thread that reads tensor memory owns one vocabulary entry and
 // sees all positions; the reduction runs over the vocabulary.  The tile is
@@ -33,8 +39,9 @@
 // four quarters are merged and the CTA writes one Partial per position; the
 // acceptance scan folds the gridDim.x partials of every row.
 //
-// Every wait is bounded: a wait that runs out records a code in *status, and
-// all roles fall through to the common exit (tensor memory is released there).
+// Every wait on a barrier is bounded: a wait that runs out records a code in
+// *status, and all roles fall through to the common exit (tensor memory is
+// released there).  No TMA load here is a multicast load.
 #pragma once
 #include <cuda.h>
 
@@ -43,17 +50,19 @@
 namespace fly {
 namespace lmhead {
 
-constexpr int kBlockV = 128;   // vocabulary entries per tile (MMA M)
+constexpr int kBlockV = 128;   // vocabulary entries per CTA and tile (the pair's MMA M is 256)
+constexpr int kPairV = 2 * kBlockV;
 constexpr int kBlockK = 64;    // hidden dims per stage: one 128-byte swizzle row of bf16
 constexpr int kMmaK = 16;      // hidden dims per tcgen05.mma (bf16)
 constexpr int kHalfN = 144;    // positions per accumulator (MMA N <= 256, multiple of 16)
 constexpr int kMaxPos = 2 * kHalfN;
 constexpr int kStagesW = 6;    // weight ring
-constexpr int kStagesH = 3;    // hidden ring
+constexpr int kStagesH = 6;    // hidden ring
 constexpr int kBytesW = kBlockK * kBlockV * 2;      // 16 KB per stage
 constexpr int kBytesWBox = kBlockK * 64 * 2;        // one TMA box: 64 entries x 64 dims
-constexpr int kBytesHHalf = kHalfN * kBlockK * 2;   // 18 KB
-constexpr int kBytesH = 2 * kBytesHHalf;
+constexpr int kBoxPos = kHalfN / 2;                 // positions per TMA box: this CTA's half of one accumulator
+constexpr int kBytesHHalf = kBoxPos * kBlockK * 2;  // 9 KB
+constexpr int kBytesH = 2 * kBytesHHalf;            // both accumulators
 constexpr int kChunk = 32;                          // positions turned through shared memory at a time
 constexpr int kChunks = kMaxPos / kChunk;           // 9
 constexpr int kTurnRow = kBlockV + 4;               // words per position row (+4: conflict-free 128-bit reads)
@@ -79,10 +88,10 @@ struct Params {
   int R;          // positions handled by this launch (1..288)
   int n0, n1;     // MMA N of the two accumulators (multiples of 16; n1 may be 0)
   int V, D;
-  int num_tiles;  // ceil(V / 128)
+  int num_tiles;  // ceil(V / 256): tiles of the CTA pairs
   int num_kb;     // ceil(D / 64)
   int row0;       // first row of this launch in hidden / partials
-  Partial* partials;  // [rows, gridDim.x]
+  Partial* partials;  // [rows, gridDim.x]: one partial state per position and CTA
   int* status;        // 0, or the code of the first wait that ran out
 };
 
@@ -99,11 +108,30 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrives on a barrier of the CTA with rank `cta` in the pair (cluster-scope release).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+// shared::cluster address of `addr` (an address in this CTA's shared memory) in the CTA of rank `cta`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t cta) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -133,9 +161,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
   return true;
 }
 
+// Tiled TMA load into THIS CTA's shared memory; the bytes are reported to `bar`, a shared::cluster
+// address that may lie in the other CTA of the pair.  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
@@ -143,19 +173,21 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem], one CTA, bf16 inputs, fp32 accumulate.
+// D[tmem] (+)= A[smem] * B[smem] over the CTA pair (M = 256: 128 rows per CTA; each CTA supplies its
+// rows of A and half of B's rows from the same shared-memory offsets), bf16 inputs, fp32 accumulate.
 __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Arrives on `bar` once every tcgen05.mma issued so far by this thread has completed.
+// Arrives on `bar` (a shared::cluster address, in either CTA of the pair) once every tcgen05.mma issued
+// so far by this thread has completed in both CTAs.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
 // 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.
@@ -182,10 +214,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
          ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: fp32 accumulator, bf16 A and B, A MN-major (vocabulary
-// contiguous), B K-major, M = 128, N = n.
+// contiguous), B K-major, M = 256 (the pair), N = n.
 __host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
-         ((uint32_t)(kBlockV >> 4) << 24);
+         ((uint32_t)(kPairV >> 4) << 24);
 }
 
 // Running statistics of one (position, vocabulary quarter) stream.
@@ -229,7 +261,7 @@ __device__ __forceinline__ void fold32(Stream& st, float (&x)[32], int v0) {
   st.u += u0 + u1;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_h,
                      const Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -246,76 +278,78 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1] epilogue go flag
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();  // 0: leader of the pair (issues the MMAs, owns the "full" barriers)
+  const int pair = (int)blockIdx.x >> 1, npairs = (int)gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStagesW; ++s) { mbar_init(full_w(s), 1); mbar_init(empty_w(s), 1); }
     for (int s = 0; s < kStagesH; ++s) { mbar_init(full_h(s), 1); mbar_init(empty_h(s), 1); }
     mbar_init(tmem_full, 1);
-    mbar_init(tmem_empty, kEpiThreads);
+    mbar_init(tmem_empty, 2 * kEpiThreads);  // the epilogue threads of both CTAs arrive on the leader's
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 0) {  // one warp allocates all of tensor memory (one CTA per SM)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffMisc),
+  if (warp == 0) {  // warp 0 of both CTAs together allocate all of tensor memory (one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + kOffMisc),
                  "r"(kTmemCols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync();  // both CTAs' barriers exist before anything is sent to them
   tc_fence_after();
   const uint32_t tmem = misc[0];
 
-  const int my_tiles = blockIdx.x < p.num_tiles ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  const int my_tiles = pair < p.num_tiles ? (p.num_tiles - 1 - pair) / npairs + 1 : 0;
 
   if (warp == 4) {
-    // ---------------- weight producer ----------------
+    // ---------------- weight producer: this CTA's 128 vocabulary entries ----------------
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        const int v0 = ((int)blockIdx.x + t * (int)gridDim.x) * kBlockV;
+        const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
           const int s = issued % kStagesW;
           const uint32_t ph = (issued / kStagesW) & 1;
           if (!mbar_wait(empty_w(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
-          mbar_expect_tx(full_w(s), kBytesW);
+          if (rank == 0) mbar_expect_tx(full_w(s), 2 * kBytesW);  // both CTAs' bytes
+          const uint32_t bar = map_to_cta(full_w(s), 0);
           const uint32_t dst = base + kOffW + s * kBytesW;
-          tma_load_2d(dst, &map_w, v0, kb * kBlockK, full_w(s));
-          tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, full_w(s));
+          tma_load_2d(dst, &map_w, v0, kb * kBlockK, bar);
+          tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, bar);
         }
       }
-      // copies still in flight must land before the CTA gives its shared memory back
-      for (int i = issued > kStagesW ? issued - kStagesW : 0; i < issued; ++i)
-        mbar_wait(full_w(i % kStagesW), (i / kStagesW) & 1, p.status, kErrTimeoutProducer);
     }
   } else if (warp == 5) {
-    // ---------------- hidden-state producer ----------------
+    // ---------------- hidden-state producer: this CTA's half of each accumulator's positions ----------------
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
       const uint32_t bytes = p.n1 > 0 ? kBytesH : kBytesHHalf;
+      const int y0 = p.row0 + (int)rank * (p.n0 / 2);
+      const int y1 = p.row0 + kHalfN + (int)rank * (p.n1 / 2);
       for (int t = 0; t < my_tiles && ok; ++t) {
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
           const int s = issued % kStagesH;
           const uint32_t ph = (issued / kStagesH) & 1;
           if (!mbar_wait(empty_h(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
-          mbar_expect_tx(full_h(s), bytes);
+          if (rank == 0) mbar_expect_tx(full_h(s), 2 * bytes);
+          const uint32_t bar = map_to_cta(full_h(s), 0);
           const uint32_t dst = base + kOffH + s * kBytesH;
-          tma_load_2d(dst, &map_h, kb * kBlockK, p.row0, full_h(s));
-          if (p.n1 > 0) tma_load_2d(dst + kBytesHHalf, &map_h, kb * kBlockK, p.row0 + kHalfN, full_h(s));
+          tma_load_2d(dst, &map_h, kb * kBlockK, y0, bar);
+          if (p.n1 > 0) tma_load_2d(dst + kBytesHHalf, &map_h, kb * kBlockK, y1, bar);
         }
       }
-      for (int i = issued > kStagesH ? issued - kStagesH : 0; i < issued; ++i)
-        mbar_wait(full_h(i % kStagesH), (i / kStagesH) & 1, p.status, kErrTimeoutProducer);
     }
   } else if (warp == 6) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (leader CTA) ----------------
+    if (lane == 0 && rank == 0) {
       const uint32_t idesc0 = instr_desc(p.n0), idesc1 = instr_desc(p.n1 > 0 ? p.n1 : 16);
       int it = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        // the epilogue must have drained the accumulators of the previous tile
+        // both epilogues must have drained the accumulators of the previous tile
         if (!mbar_wait(tmem_empty, (t & 1) ^ 1, p.status, kErrTimeoutMma)) break;
         tc_fence_after();
         for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
@@ -342,10 +376,16 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
               mma_bf16(tmem + kHalfN, da, db1, idesc1, acc);
             }
           }
-          mma_commit(empty_w(sw));  // the stage may be refilled once these MMAs have read it
+          // the stage may be refilled, in both CTAs, once these MMAs have read it
+          mma_commit(empty_w(sw));
+          mma_commit(map_to_cta(empty_w(sw), 1));
           mma_commit(empty_h(sh));
+          mma_commit(map_to_cta(empty_h(sh), 1));
         }
-        if (ok) mma_commit(tmem_full);
+        if (ok) {
+          mma_commit(tmem_full);
+          mma_commit(map_to_cta(tmem_full, 1));
+        }
       }
     }
   } else {
@@ -357,13 +397,12 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     const int nchunks = (p.R + kChunk - 1) / kChunk;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     for (int t = 0; t < my_tiles; ++t) {
-      const int tile = (int)blockIdx.x + t * (int)gridDim.x;
       if (threadIdx.x == 0) misc[1] = mbar_wait(tmem_full, t & 1, p.status, kErrTimeoutEpilogue) ? 1u : 0u;
       epi_bar();
       const bool go = misc[1] != 0;  // one thread waits, all take the same decision
       if (!go) break;
       tc_fence_after();
-      const int v0 = tile * kBlockV + warp * 32;
+      const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + warp * 32;
       const int limit = p.V - v0;  // entries of this quarter that exist
 #pragma unroll
       for (int c = 0; c < kChunks; ++c) {
@@ -372,7 +411,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
           tmem_ld32(tmem + lane_base + (uint32_t)(c * kChunk), r);
           if (c == nchunks - 1) {  // last read of this tile: hand the accumulators back to the MMA issuer
             tc_fence_before();
-            mbar_arrive(tmem_empty);
+            mbar_arrive_remote(map_to_cta(tmem_empty, 0));
           }
           epi_bar();  // everyone is done reading the previous block
 #pragma unroll
@@ -414,11 +453,18 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     }
   }
 
+  // Common exit.  After a failed wait give stragglers (TMA copies still in flight towards this
+  // CTA's shared memory) time to land before the shared memory is handed back.
+  if (*(volatile int*)p.status != 0) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 2000000ull) {}
+  }
   tc_fence_before();
   __syncthreads();
+  cluster_sync();  // neither CTA leaves while its partner may still signal its barriers or read its operands
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
 }
 
