@@ -56,8 +56,7 @@ constexpr int kBlockK = 64;    // hidden dims per stage: one 128-byte swizzle ro
 constexpr int kMmaK = 16;      // hidden dims per tcgen05.mma (bf16)
 constexpr int kHalfN = 144;    // positions per accumulator (MMA N <= 256, multiple of 16)
 constexpr int kMaxPos = 2 * kHalfN;
-constexpr int kStagesW = 6;    // weight ring
-constexpr int kStagesH = 6;    // hidden ring
+constexpr int kStages = 6;     // operand ring: one stage = one 64-dim slice of the weight tile and of the hidden tile
 constexpr int kBytesW = kBlockK * kBlockV * 2;      // 16 KB per stage
 constexpr int kBytesWBox = kBlockK * 64 * 2;        // one TMA box: 64 entries x 64 dims
 constexpr int kBoxPos = kHalfN / 2;                 // positions per TMA box: this CTA's half of one accumulator
@@ -72,14 +71,14 @@ constexpr int kThreads = 224;
 constexpr int kTmemCols = 512;
 
 constexpr int kOffW = 0;
-constexpr int kOffH = kOffW + kStagesW * kBytesW;
-constexpr int kOffTurn = kOffH + kStagesH * kBytesH;
+constexpr int kOffH = kOffW + kStages * kBytesW;
+constexpr int kOffTurn = kOffH + kStages * kBytesH;
 constexpr int kOffBar = kOffTurn + kTurnBytes;
-constexpr int kNumBars = 2 * kStagesW + 2 * kStagesH + 2;
+constexpr int kNumBars = 2 * kStages + 2;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;
 constexpr int kSmemBytes = kOffMisc + 32 + 1024;    // + slack to align the base to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-static_assert(kMaxPos * 4 * 16 <= kStagesW * kBytesW, "final merge buffer reuses the weight ring");
+static_assert(kMaxPos * 4 * 16 <= kStages * kBytesW, "final merge buffer reuses the weight ring");
 
 constexpr int kErrTimeoutProducer = 1, kErrTimeoutMma = 2, kErrTimeoutEpilogue = 3;
 constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;  // far above any legitimate wait (a tile takes ~50 us)
@@ -269,11 +268,12 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;  // swizzle atoms are 1024-byte aligned
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t bar0 = base + kOffBar;
-  auto full_w = [&](int s) { return bar0 + 8u * s; };
-  auto empty_w = [&](int s) { return bar0 + 8u * (kStagesW + s); };
-  auto full_h = [&](int s) { return bar0 + 8u * (2 * kStagesW + s); };
-  auto empty_h = [&](int s) { return bar0 + 8u * (2 * kStagesW + kStagesH + s); };
-  const uint32_t tmem_full = bar0 + 8u * (2 * kStagesW + 2 * kStagesH);
+  // full(s), in the leader: the stage's operands of BOTH CTAs have landed (the leader's two producers
+  // arrive with the expected byte counts; every TMA load of the pair reports its bytes here).
+  // empty(s), in each CTA: the MMAs that read the stage have completed, the producers may refill it.
+  auto full = [&](int s) { return bar0 + 8u * s; };
+  auto empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+  const uint32_t tmem_full = bar0 + 8u * (2 * kStages);
   const uint32_t tmem_empty = tmem_full + 8u;
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1] epilogue go flag
 
@@ -282,8 +282,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   const int pair = (int)blockIdx.x >> 1, npairs = (int)gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStagesW; ++s) { mbar_init(full_w(s), 1); mbar_init(empty_w(s), 1); }
-    for (int s = 0; s < kStagesH; ++s) { mbar_init(full_h(s), 1); mbar_init(empty_h(s), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 2); mbar_init(empty(s), 1); }
     mbar_init(tmem_full, 1);
     mbar_init(tmem_empty, 2 * kEpiThreads);  // the epilogue threads of both CTAs arrive on the leader's
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -310,11 +309,11 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
-          const int s = issued % kStagesW;
-          const uint32_t ph = (issued / kStagesW) & 1;
-          if (!mbar_wait(empty_w(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(full_w(s), 2 * kBytesW);  // both CTAs' bytes
-          const uint32_t bar = map_to_cta(full_w(s), 0);
+          const int s = issued % kStages;
+          const uint32_t ph = (issued / kStages) & 1;
+          if (!mbar_wait(empty(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full(s), 2 * kBytesW);  // both CTAs' bytes
+          const uint32_t bar = map_to_cta(full(s), 0);
           const uint32_t dst = base + kOffW + s * kBytesW;
           tma_load_2d(dst, &map_w, v0, kb * kBlockK, bar);
           tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, bar);
@@ -331,11 +330,11 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       const int y1 = p.row0 + kHalfN + (int)rank * (p.n1 / 2);
       for (int t = 0; t < my_tiles && ok; ++t) {
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
-          const int s = issued % kStagesH;
-          const uint32_t ph = (issued / kStagesH) & 1;
-          if (!mbar_wait(empty_h(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(full_h(s), 2 * bytes);
-          const uint32_t bar = map_to_cta(full_h(s), 0);
+          const int s = issued % kStages;
+          const uint32_t ph = (issued / kStages) & 1;
+          if (!mbar_wait(empty(s), ph ^ 1, p.status, kErrTimeoutProducer)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full(s), 2 * bytes);
+          const uint32_t bar = map_to_cta(full(s), 0);
           const uint32_t dst = base + kOffH + s * kBytesH;
           tma_load_2d(dst, &map_h, kb * kBlockK, y0, bar);
           if (p.n1 > 0) tma_load_2d(dst + kBytesHHalf, &map_h, kb * kBlockK, y1, bar);
@@ -346,22 +345,22 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     // ---------------- MMA issuer (leader CTA) ----------------
     if (lane == 0 && rank == 0) {
       const uint32_t idesc0 = instr_desc(p.n0), idesc1 = instr_desc(p.n1 > 0 ? p.n1 : 16);
-      int it = 0;
+      uint32_t peer_empty[kStages];
+#pragma unroll
+      for (int s = 0; s < kStages; ++s) peer_empty[s] = map_to_cta(empty(s), 1);
+      const uint32_t peer_tmem_full = map_to_cta(tmem_full, 1);
+      int it = 0, st = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
         // both epilogues must have drained the accumulators of the previous tile
         if (!mbar_wait(tmem_empty, (t & 1) ^ 1, p.status, kErrTimeoutMma)) break;
         tc_fence_after();
         for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
-          const int sw = it % kStagesW, sh = it % kStagesH;
-          if (!mbar_wait(full_w(sw), (it / kStagesW) & 1, p.status, kErrTimeoutMma) ||
-              !mbar_wait(full_h(sh), (it / kStagesH) & 1, p.status, kErrTimeoutMma)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t aw = base + kOffW + sw * kBytesW;
-          const uint32_t bh = base + kOffH + sh * kBytesH;
+          // TMA-written operands need no tcgen05 fence: the barrier wait orders them before the MMAs
+          if (!mbar_wait(full(st), ph, p.status, kErrTimeoutMma)) { ok = false; break; }
+          const uint32_t aw = base + kOffW + st * kBytesW;
+          const uint32_t bh = base + kOffH + st * kBytesH;
 #pragma unroll
           for (int ks = 0; ks < kBlockK / kMmaK; ++ks) {
             // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden
@@ -377,14 +376,16 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             }
           }
           // the stage may be refilled, in both CTAs, once these MMAs have read it
-          mma_commit(empty_w(sw));
-          mma_commit(map_to_cta(empty_w(sw), 1));
-          mma_commit(empty_h(sh));
-          mma_commit(map_to_cta(empty_h(sh), 1));
+          mma_commit(empty(st));
+          uint32_t pe = peer_empty[0];
+#pragma unroll
+          for (int s = 1; s < kStages; ++s) pe = st == s ? peer_empty[s] : pe;
+          mma_commit(pe);
+          if (++st == kStages) { st = 0; ph ^= 1; }
         }
         if (ok) {
           mma_commit(tmem_full);
-          mma_commit(map_to_cta(tmem_full, 1));
+          mma_commit(peer_tmem_full);
         }
       }
     }
