@@ -24,7 +24,8 @@
 //
 // Pairs are persistent: pair i walks vocabulary tiles i, i + #pairs, ...  Warp
 // roles in each CTA: 0-3 epilogue (they own the four 32-lane quarters of tensor
-// memory), 4 weight producer, 5 hidden producer, 6 MMA issuer (leader CTA only).
+// memory), 4 weight producer, 5 hidden producer, 6 and 7 MMA issuers (leader CTA
+// only; one per accumulator).
 // "Full" barriers live in the leader: both CTAs' TMA loads report their bytes
 // there.  The leader's tcgen05.commit releases a stage in both CTAs.
 //
@@ -67,7 +68,7 @@ constexpr int kChunks = kMaxPos / kChunk;           // 9
 constexpr int kTurnRow = kBlockV + 4;               // words per position row (+4: conflict-free 128-bit reads)
 constexpr int kTurnBytes = kChunk * kTurnRow * 4;
 constexpr int kEpiThreads = 128;
-constexpr int kThreads = 224;
+constexpr int kThreads = 256;
 constexpr int kTmemCols = 512;
 
 constexpr int kOffW = 0;
@@ -174,13 +175,17 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 
 // D[tmem] (+)= A[smem] * B[smem] over the CTA pair (M = 256: 128 rows per CTA; each CTA supplies its
 // rows of A and half of B's rows from the same shared-memory offsets), bf16 inputs, fp32 accumulate.
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                         uint32_t accumulate) {
+// The shared-memory descriptors are passed as (low word, high word): only the low word (start
+// address) changes from one MMA to the next.
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                         uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // Arrives on `bar` (a shared::cluster address, in either CTA of the pair) once every tcgen05.mma issued
@@ -206,12 +211,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ---- descriptors ---------------------------------------------------------------
-// Shared-memory matrix descriptor of tcgen05.mma: start address, leading and
-// stride byte offsets in 16-byte units, descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
-         ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
+// Shared-memory matrix descriptor of tcgen05.mma (64 bits).  Low word: start address and leading
+// byte offset, both in 16-byte units.  High word: stride byte offset in 16-byte units, descriptor
+// version 1, 128-byte swizzle.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr >> 4) & 0x3fffu) | (((lbo_bytes >> 4) & 0x3fffu) << 16);
 }
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);  // groups of 8 rows 1024 bytes apart
 // Instruction descriptor: fp32 accumulator, bf16 A and B, A MN-major (vocabulary
 // contiguous), B K-major, M = 256 (the pair), N = n.
 __host__ __device__ constexpr uint32_t instr_desc(int n) {
@@ -282,8 +288,9 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   const int pair = (int)blockIdx.x >> 1, npairs = (int)gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 2); mbar_init(empty(s), 1); }
-    mbar_init(tmem_full, 1);
+    const uint32_t issuers = p.n1 > 0 ? 2 : 1;  // one MMA-issuing thread per accumulator
+    for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 2); mbar_init(empty(s), issuers); }
+    mbar_init(tmem_full, issuers);
     mbar_init(tmem_empty, 2 * kEpiThreads);  // the epilogue threads of both CTAs arrive on the leader's
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -341,51 +348,48 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         }
       }
     }
-  } else if (warp == 6) {
-    // ---------------- MMA issuer (leader CTA) ----------------
-    if (lane == 0 && rank == 0) {
-      const uint32_t idesc0 = instr_desc(p.n0), idesc1 = instr_desc(p.n1 > 0 ? p.n1 : 16);
-      uint32_t peer_empty[kStages];
-#pragma unroll
-      for (int s = 0; s < kStages; ++s) peer_empty[s] = map_to_cta(empty(s), 1);
-      const uint32_t peer_tmem_full = map_to_cta(tmem_full, 1);
-      int it = 0, st = 0;
+  } else if (warp >= 6) {
+    // ---------------- MMA issuers (leader CTA): warp 6 feeds accumulator 0, warp 7 accumulator 1 ----------------
+    // One thread cannot issue MMAs, commits and barrier waits fast enough to keep the tensor pipe
+    // busy with two 144-column MMAs per 16 hidden dims, so each accumulator has an issuer of its own.
+    const int half = warp - 6;
+    if (lane == 0 && rank == 0 && (half == 0 || p.n1 > 0)) {
+      const uint32_t idesc = instr_desc(half == 0 ? p.n0 : p.n1);
+      const uint32_t d_tmem = tmem + (uint32_t)(half * kHalfN);
+      // Everything that changes from one MMA to the next is a 32-bit add: this thread has to issue one
+      // MMA every ~70 cycles, so the loop is kept to a few instructions per MMA.
+      // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden dims
+      // 1024 bytes apart (stride offset); 16 hidden dims further = 16 rows of 128 bytes.
+      // B, K-major: groups of 8 positions 1024 bytes apart; 16 hidden dims further = 32 bytes.
+      const uint32_t a_lo0 = desc_lo(base + kOffW, kBytesWBox);
+      const uint32_t b_lo0 = desc_lo(base + kOffH + half * kBytesHHalf, 16);
+      const uint32_t peer_delta = map_to_cta(bar0, 1) - bar0;  // same offset in the partner's shared memory
+      int st = 0;
       uint32_t ph = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
         // both epilogues must have drained the accumulators of the previous tile
         if (!mbar_wait(tmem_empty, (t & 1) ^ 1, p.status, kErrTimeoutMma)) break;
         tc_fence_after();
-        for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+        for (int kb = 0; kb < p.num_kb; ++kb) {
           // TMA-written operands need no tcgen05 fence: the barrier wait orders them before the MMAs
           if (!mbar_wait(full(st), ph, p.status, kErrTimeoutMma)) { ok = false; break; }
-          const uint32_t aw = base + kOffW + st * kBytesW;
-          const uint32_t bh = base + kOffH + st * kBytesH;
+          const uint32_t a_lo = a_lo0 + (uint32_t)st * (kBytesW >> 4);
+          const uint32_t b_lo = b_lo0 + (uint32_t)st * (kBytesH >> 4);
 #pragma unroll
           for (int ks = 0; ks < kBlockK / kMmaK; ++ks) {
-            // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden
-            // dims 1024 bytes apart (stride offset); 16 hidden dims further = 16 rows of 128 bytes.
-            const uint64_t da = smem_desc(aw + ks * (kMmaK * 128), kBytesWBox, 1024);
-            // B, K-major: groups of 8 positions 1024 bytes apart; 16 hidden dims further = 32 bytes.
-            const uint64_t db0 = smem_desc(bh + ks * (kMmaK * 2), 16, 1024);
-            const uint32_t acc = (kb | ks) != 0;
-            mma_bf16(tmem, da, db0, idesc0, acc);
-            if (p.n1 > 0) {
-              const uint64_t db1 = smem_desc(bh + kBytesHHalf + ks * (kMmaK * 2), 16, 1024);
-              mma_bf16(tmem + kHalfN, da, db1, idesc1, acc);
-            }
+            const uint32_t acc = ks == 0 ? (uint32_t)(kb != 0) : 1u;
+            mma_bf16(d_tmem, a_lo + ks * ((kMmaK * 128) >> 4), b_lo + ks * ((kMmaK * 2) >> 4), kDescHi, idesc, acc);
           }
           // the stage may be refilled, in both CTAs, once these MMAs have read it
-          mma_commit(empty(st));
-          uint32_t pe = peer_empty[0];
-#pragma unroll
-          for (int s = 1; s < kStages; ++s) pe = st == s ? peer_empty[s] : pe;
-          mma_commit(pe);
+          const uint32_t eb = empty(st);
+          mma_commit(eb);
+          mma_commit(eb + peer_delta);
           if (++st == kStages) { st = 0; ph ^= 1; }
         }
         if (ok) {
           mma_commit(tmem_full);
-          mma_commit(peer_tmem_full);
+          mma_commit(tmem_full + peer_delta);
         }
       }
     }
