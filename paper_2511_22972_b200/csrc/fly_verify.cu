@@ -50,7 +50,8 @@ struct fly_verify {
   int last_launches = 0;
   int last_cuda_error = 0;
   // fused LM-head path (cfg.hidden > 0)
-  fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]
+  fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]: one partial state per row and CTA
+  fly::Partial* lm_folded = nullptr;    // [max_rows]: the same, folded over the CTAs
   int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
   int lm_pairs = 0;                     // CTA pairs that can be resident at once
   PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
@@ -238,8 +239,18 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
   }
-  const fly::ScanParams sp = scan_params(h, a, h->lm_partials, grid);
-  cudaError_t e = launch_scan(sp, st);
+  cudaError_t e;
+  {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    const unsigned warps = fly::kFoldThreads / 32;
+    fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, true);
+    e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->lm_partials, grid, h->lm_folded, (int)rows);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches++;
+  }
+  const fly::ScanParams sp = scan_params(h, a, h->lm_folded, 1);
+  e = launch_scan(sp, st);
   if (e != cudaSuccess) return cuda_fail(h, e);
   h->last_launches++;
   return FLY_OK;
@@ -313,6 +324,7 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   if (e != cudaSuccess) { cudaFree(h->partials); cudaFree(h->tickets); delete h; return FLY_ERR_CUDA; }
   if (c->hidden > 0) {
     e = cudaMalloc(&h->lm_partials, (size_t)h->max_rows * h->sm_count * sizeof(fly::Partial));
+    if (e == cudaSuccess) e = cudaMalloc(&h->lm_folded, (size_t)h->max_rows * sizeof(fly::Partial));
     if (e == cudaSuccess) e = cudaMalloc(&h->lm_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->lm_status, 0, sizeof(int));
     if (e == cudaSuccess)
@@ -344,7 +356,8 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
     if (e != cudaSuccess || !fn) {
       fly_status_t st = cuda_fail(h, e);
       (void)st;
-      cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_partials); cudaFree(h->lm_status);
+      cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_partials); cudaFree(h->lm_folded);
+      cudaFree(h->lm_status);
       delete h;
       return FLY_ERR_CUDA;
     }
@@ -361,6 +374,7 @@ fly_status_t fly_verify_destroy(fly_verify_t* h) {
     cudaFree(h->partials);
     cudaFree(h->tickets);
     cudaFree(h->lm_partials);
+    cudaFree(h->lm_folded);
     cudaFree(h->lm_status);
     cudaFree(h->st_hidden);
     cudaFree(h->st_logits);
