@@ -86,21 +86,13 @@ __device__ __forceinline__ uint32_t bf2_max_nan(uint32_t a, uint32_t b) {
   return d;
 }
 
-// One warp slice of UNROLL*32 segments of bf16 logits.  seg0 = index of the
-// slice's first segment inside the row, seg_end = end of this unit's range.
+constexpr uint32_t kNegInf2 = 0xff80ff80u;  // bf16 (-inf, -inf)
+
+// Folds one warp slice of UNROLL*32 segments of bf16 logits, already in registers, into the
+// warp's running state.  w[j] is segment seg0 + j*32 + lane of the row (8 logits).
 template <int UNROLL>
-__device__ __forceinline__ void warp_slice_bf16(WarpAcc& a, const uint4* __restrict__ row, int seg0,
-                                                int seg_end, int lane) {
-  constexpr uint32_t kNegInf2 = 0xff80ff80u;  // (-inf, -inf)
+__device__ __forceinline__ void fold_slice_bf16(WarpAcc& a, uint32_t (&w)[UNROLL][4], int seg0, int lane) {
   constexpr uint32_t kFloor2 = 0xc974c974u;   // bf16(kMaskFloor) twice
-  uint32_t w[UNROLL][4];
-#pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    const int s = seg0 + j * 32 + lane;
-    uint4 q = make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
-    if (s < seg_end) q = ld_stream(row + s);
-    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-  }
   // clamp masked entries to the floor (NaN survives the clamp and ends in S)
   uint32_t lm2 = kFloor2;
 #pragma unroll
@@ -137,18 +129,25 @@ __device__ __forceinline__ void warp_slice_bf16(WarpAcc& a, const uint4* __restr
     }
 }
 
+// One warp slice of UNROLL*32 segments of bf16 logits read from global memory.  seg0 = index of
+// the slice's first segment inside the row, seg_end = end of this unit's range.
 template <int UNROLL>
-__device__ __forceinline__ void warp_slice_f32(WarpAcc& a, const uint4* __restrict__ row, int seg0,
-                                               int seg_end, int lane) {
-  float x[UNROLL][4];
+__device__ __forceinline__ void warp_slice_bf16(WarpAcc& a, const uint4* __restrict__ row, int seg0,
+                                                int seg_end, int lane) {
+  uint32_t w[UNROLL][4];
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j) {
     const int s = seg0 + j * 32 + lane;
-    uint4 q = make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+    uint4 q = make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
     if (s < seg_end) q = ld_stream(row + s);
-    x[j][0] = __uint_as_float(q.x); x[j][1] = __uint_as_float(q.y);
-    x[j][2] = __uint_as_float(q.z); x[j][3] = __uint_as_float(q.w);
+    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
   }
+  fold_slice_bf16<UNROLL>(a, w, seg0, lane);
+}
+
+// The same for fp32 logits: x[j] is segment seg0 + j*32 + lane of the row (4 logits).
+template <int UNROLL>
+__device__ __forceinline__ void fold_slice_f32(WarpAcc& a, float (&x)[UNROLL][4], int seg0, int lane) {
   float lm = kMaskFloor;
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j)
@@ -178,6 +177,21 @@ __device__ __forceinline__ void warp_slice_f32(WarpAcc& a, const uint4* __restri
     acc_add(x[j][2], nr, a.S0, a.u0);
     acc_add(x[j][3], nr, a.S1, a.u1);
   }
+}
+
+template <int UNROLL>
+__device__ __forceinline__ void warp_slice_f32(WarpAcc& a, const uint4* __restrict__ row, int seg0,
+                                               int seg_end, int lane) {
+  float x[UNROLL][4];
+#pragma unroll
+  for (int j = 0; j < UNROLL; ++j) {
+    const int s = seg0 + j * 32 + lane;
+    uint4 q = make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
+    if (s < seg_end) q = ld_stream(row + s);
+    x[j][0] = __uint_as_float(q.x); x[j][1] = __uint_as_float(q.y);
+    x[j][2] = __uint_as_float(q.z); x[j][3] = __uint_as_float(q.w);
+  }
+  fold_slice_f32<UNROLL>(a, x, seg0, lane);
 }
 
 // Element-wise slice for rows without 16-byte structure and for the ragged
