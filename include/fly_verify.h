@@ -166,7 +166,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* 
  * The first call on each device looks up the device address of the built-in
  * array (which also makes the CUDA runtime load the library's device code).
  * Make that first call outside any stream capture; later calls only enqueue
- * work on `cuda_stream` (one small memset of the arrival counters, one kernel).
+ * work on `cuda_stream` (one 4 KB memset of the arrival counters, one kernel).
  *
  * All calls on a device share the one array, and it keeps whatever the last
  * call left there.  The counters are cleared on the stream at the start of
@@ -176,7 +176,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* 
  * scratch and corrupt each other: serialise them, e.g. keep them on one stream. */
 #define FLY_STATIC_MAX_BATCH 1024
 #define FLY_STATIC_MAX_PIECES 16384
-#define FLY_STATIC_SCRATCH_BYTES (FLY_STATIC_MAX_BATCH * 4 + 256 + FLY_STATIC_MAX_PIECES * 16) /* 260.25 KiB */
+#define FLY_STATIC_SCRATCH_BYTES (FLY_STATIC_MAX_BATCH * 4 + FLY_STATIC_MAX_PIECES * 16) /* 260 KiB */
 fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t logits_dtype,
                                    const fly_verify_args_t* args, void* cuda_stream);
 
@@ -193,16 +193,11 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
  *                         kernel is still draining and waits for it to complete only before its
  *                         first write.  Only correct if the logits of this step were complete
  *                         before that previous kernel started (e.g. back-to-back steps over inputs
- *                         already in memory).  0 (default): plain stream order.
- * FLY_OPT_KERNEL_FORM     0 (default): rows of at least 32 KB with 16-byte structure are reduced by the
- *                         persistent streaming kernel (one CTA per SM, logits staged through shared
- *                         memory by bulk asynchronous copies); everything else by one thread block per
- *                         (row, piece).  1: one thread block per (row, piece) always. */
+ *                         already in memory).  0 (default): plain stream order. */
 typedef enum {
   FLY_OPT_SPLITS = 0,
   FLY_OPT_SCAN_MODE = 1,
-  FLY_OPT_STREAM_OVERLAP = 2,
-  FLY_OPT_KERNEL_FORM = 3
+  FLY_OPT_STREAM_OVERLAP = 2
 } fly_option_t;
 fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
 

@@ -17,7 +17,7 @@ FLY_STATIC_MAX_BATCH, FLY_STATIC_MAX_PIECES = 1024, 16384
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
-FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP, FLY_OPT_KERNEL_FORM = range(4)
+FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
@@ -140,9 +140,6 @@ class FlyVerify:
 
     def set_scan_mode(self, separate_kernel: bool):
         self.set_option(FLY_OPT_SCAN_MODE, 1 if separate_kernel else 0)
-
-    def set_kernel_form(self, block_per_piece: bool):
-        self.set_option(FLY_OPT_KERNEL_FORM, 1 if block_per_piece else 0)
 
     def set_stream_overlap(self, on: bool):
         self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)

@@ -15,11 +15,14 @@
 #include "lmhead_kernel.cuh"
 #include "reduce_kernel.cuh"
 #include "scan_kernel.cuh"
-#include "stream_kernel.cuh"
 
 namespace {
 
 constexpr int kMaxSplits = 32;
+// 16-byte loads in flight per lane and slice in the row-reduction kernel.  Measured: 2 and 8 are
+// slower than 4, and loading the next slice before folding the current one (two register sets)
+// changes nothing.
+constexpr int kReduceUnroll = 4;
 constexpr int kMaxK = 63;
 
 struct DeviceGuard {
@@ -46,7 +49,6 @@ struct fly_verify {
   unsigned int* tickets = nullptr;   // [max_batch], zero between launches
   int forced_splits = 0;
   int scan_mode = 0;   // 0: fused tail, 1: separate kernel
-  int kernel_form = 0; // 0: streaming kernel where it applies, 1: one block per (row, piece) always
   int overlap = 0;
   int last_splits = 1;
   int last_launches = 0;
@@ -54,8 +56,7 @@ struct fly_verify {
   // fused LM-head path (cfg.hidden > 0)
   fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]: one partial state per row and CTA
   fly::Partial* lm_folded = nullptr;    // [max_rows]: the same, folded over the CTAs
-  int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read);
-                                        // shared by the fused path and the streaming row reduction
+  int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
   int lm_pairs = 0;                     // CTA pairs that can be resident at once
   PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
   CUtensorMap map_w, map_h;             // cached for (map_w_ptr, map_h_ptr, map_h_rows)
@@ -114,40 +115,6 @@ int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t ma
   return (int)cap;
 }
 
-// Pieces per row for the persistent streaming kernel: CTA c walks units [c*U/G, (c+1)*U/G), so what
-// matters is how evenly U = rows * pieces divides among the G CTAs.  The smallest piece count within
-// 1% of the best balance wins (a unit end costs a block-wide merge), with pieces of at least 32 KB.
-int stream_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
-  const int64_t G = h->sm_count;
-  int64_t cap = row_bytes / 32768;
-  if (cap < 1) cap = 1;
-  if (cap > kMaxSplits) cap = kMaxSplits;
-  if (cap > max_pieces) cap = max_pieces;
-  double best = 0.0;
-  for (int64_t s = 1; s <= cap; ++s) {
-    const int64_t n = rows * s;
-    const double bal = (double)n / (double)(G * ((n + G - 1) / G));
-    if (bal > best) best = bal;
-  }
-  for (int64_t s = 1; s <= cap; ++s) {
-    const int64_t n = rows * s;
-    const double bal = (double)n / (double)(G * ((n + G - 1) / G));
-    if (bal >= best - 0.01) return (int)s;
-  }
-  return (int)cap;
-}
-
-// Once per device (with that device current): the streaming kernel needs more dynamic shared memory
-// than the default limit.
-cudaError_t stream_kernel_setup() {
-  cudaError_t e = cudaFuncSetAttribute(fly::stream::reduce_rows_stream<__nv_bfloat16>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, fly::stream::kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fly::stream::reduce_rows_stream<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             fly::stream::kSmemBytes);
-  return e;
-}
-
 void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned grid, unsigned block, cudaStream_t st,
                  bool programmatic) {
   memset(cfg, 0, sizeof(*cfg));
@@ -164,36 +131,11 @@ void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned gr
 template <typename T>
 cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_stride, int V, int64_t rows,
                           int forced, fly::Partial* partials, cudaStream_t st, int* splits_out,
-                          fly::ScanParams tail, bool overlap, int* status) {
+                          fly::ScanParams tail, bool overlap) {
   constexpr int kE = fly::Seg<T>::kElems;
   const bool vec = ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
                    (V >= kE * 32);
   const int64_t row_bytes = (int64_t)V * (int64_t)sizeof(T);
-  if (vec && h->kernel_form != 1 && row_bytes >= 2 * fly::stream::kChunkBytes) {
-    // persistent streaming kernel (TMA bulk copies through a shared-memory ring)
-    namespace R = fly::stream;
-    const int nseg = V / kE;
-    int splits = forced > 0 ? forced : stream_splits(h, rows, row_bytes, nseg / R::kChunkSegs);
-    if (splits > nseg) splits = nseg;
-    R::Params p;
-    p.logits = logits;
-    p.row_stride = row_stride;
-    p.V = V;
-    p.nseg = nseg;
-    p.splits = splits;
-    p.segs_per_split = (nseg + splits - 1) / splits;
-    p.units = (int)(rows * splits);
-    p.partials = partials;
-    p.status = status;
-    *splits_out = splits;
-    tail.splits = splits;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    const unsigned grid = (unsigned)(p.units < h->sm_count ? p.units : h->sm_count);
-    fill_launch(&cfg, attr, grid, R::kThreads, st, overlap);
-    cfg.dynamicSmemBytes = R::kSmemBytes;
-    return cudaLaunchKernelEx(&cfg, R::reduce_rows_stream<T>, p, tail);
-  }
   if (vec) {
     const int nseg = V / kE;
     int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, nseg);
@@ -204,7 +146,7 @@ cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_s
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     fill_launch(&cfg, attr, (unsigned)(rows * splits), fly::kReduceThreads, st, overlap);
-    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_vec<T, 4>, static_cast<const T*>(logits), row_stride, V, nseg,
+    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_vec<T, kReduceUnroll>, static_cast<const T*>(logits), row_stride, V, nseg,
                               splits, segs_per_split, partials, tail);
   } else {
     int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, (V + 31) / 32);
@@ -385,7 +327,6 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   if (e == cudaSuccess) e = cudaMemset(h->tickets, 0, (size_t)c->max_batch * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->lm_status, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(h->lm_status, 0, sizeof(int));
-  if (e == cudaSuccess) e = stream_kernel_setup();
   if (e != cudaSuccess) { cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_status); delete h; return FLY_ERR_CUDA; }
   if (c->hidden > 0) {
     e = cudaMalloc(&h->lm_partials, (size_t)h->max_rows * h->sm_count * sizeof(fly::Partial));
@@ -463,10 +404,6 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->overlap = v;
       return FLY_OK;
-    case FLY_OPT_KERNEL_FORM:
-      if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
-      h->kernel_form = v;
-      return FLY_OK;
   }
   return FLY_ERR_INVALID_ARG;
 }
@@ -531,10 +468,10 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
     int splits = 1;
     if (h->cfg.logits_dtype == FLY_BF16)
       e = launch_reduce<__nv_bfloat16>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
-                                       h->overlap != 0, h->lm_status);
+                                       h->overlap != 0);
     else
       e = launch_reduce<float>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
-                               h->overlap != 0, h->lm_status);
+                               h->overlap != 0);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
     h->last_splits = splits;
@@ -663,8 +600,6 @@ cudaError_t static_scratch_for(int device, StaticSlot* out) {
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
     if (e != cudaSuccess) return e;
     s.sm_count = sms > 0 ? sms : 148;
-    e = stream_kernel_setup();
-    if (e != cudaSuccess) return e;
     s.base = p;
   }
   *out = s;
@@ -695,11 +630,9 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
   if (!g.ok) return FLY_ERR_CUDA;
   StaticSlot slot;
   if (static_scratch_for(device, &slot) != cudaSuccess) return FLY_ERR_CUDA;
-  // layout of the array: arrival counters | status word of the kernels' bounded waits (256-byte slot) | partial states
   unsigned int* tickets = static_cast<unsigned int*>(slot.base);
-  int* status = reinterpret_cast<int*>(static_cast<unsigned char*>(slot.base) + FLY_STATIC_MAX_BATCH * 4);
   fly::Partial* partials =
-      reinterpret_cast<fly::Partial*>(static_cast<unsigned char*>(slot.base) + FLY_STATIC_MAX_BATCH * 4 + 256);
+      reinterpret_cast<fly::Partial*>(static_cast<unsigned char*>(slot.base) + FLY_STATIC_MAX_BATCH * 4);
   h.sm_count = slot.sm_count;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -727,13 +660,13 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
   p.row_flags = a->row_flags;
 
   // The arrival counters must start at zero, whatever an earlier call left behind.
-  cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4 + 256, st);
+  cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4, st);
   if (e != cudaSuccess) return FLY_ERR_CUDA;
   int used = 1;
   if (logits_dtype == FLY_BF16)
-    e = launch_reduce<__nv_bfloat16>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false, status);
+    e = launch_reduce<__nv_bfloat16>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
   else
-    e = launch_reduce<float>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false, status);
+    e = launch_reduce<float>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
   return e == cudaSuccess ? FLY_OK : FLY_ERR_CUDA;
 }
 

@@ -129,21 +129,6 @@ __device__ __forceinline__ void fold_slice_bf16(WarpAcc& a, uint32_t (&w)[UNROLL
     }
 }
 
-// One warp slice of UNROLL*32 segments of bf16 logits read from global memory.  seg0 = index of
-// the slice's first segment inside the row, seg_end = end of this unit's range.
-template <int UNROLL>
-__device__ __forceinline__ void warp_slice_bf16(WarpAcc& a, const uint4* __restrict__ row, int seg0,
-                                                int seg_end, int lane) {
-  uint32_t w[UNROLL][4];
-#pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    const int s = seg0 + j * 32 + lane;
-    uint4 q = make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
-    if (s < seg_end) q = ld_stream(row + s);
-    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-  }
-  fold_slice_bf16<UNROLL>(a, w, seg0, lane);
-}
 
 // The same for fp32 logits: x[j] is segment seg0 + j*32 + lane of the row (4 logits).
 template <int UNROLL>
@@ -179,19 +164,41 @@ __device__ __forceinline__ void fold_slice_f32(WarpAcc& a, float (&x)[UNROLL][4]
   }
 }
 
+
+// Loads segments seg0 + j*32 + lane (j < UNROLL) of a row into registers; segments at or past
+// seg_end read as -inf.  A full slice takes the unpredicated path.
 template <int UNROLL>
-__device__ __forceinline__ void warp_slice_f32(WarpAcc& a, const uint4* __restrict__ row, int seg0,
-                                               int seg_end, int lane) {
-  float x[UNROLL][4];
+__device__ __forceinline__ void load_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ row, int seg0,
+                                           int seg_end, int lane, uint32_t fill) {
+  if (seg0 + UNROLL * 32 <= seg_end) {
 #pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    const int s = seg0 + j * 32 + lane;
-    uint4 q = make_uint4(0xff800000u, 0xff800000u, 0xff800000u, 0xff800000u);
-    if (s < seg_end) q = ld_stream(row + s);
-    x[j][0] = __uint_as_float(q.x); x[j][1] = __uint_as_float(q.y);
-    x[j][2] = __uint_as_float(q.z); x[j][3] = __uint_as_float(q.w);
+    for (int j = 0; j < UNROLL; ++j) {
+      const uint4 q = ld_stream(row + seg0 + j * 32 + lane);
+      w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j) {
+      const int s = seg0 + j * 32 + lane;
+      uint4 q = make_uint4(fill, fill, fill, fill);
+      if (s < seg_end) q = ld_stream(row + s);
+      w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
+    }
   }
-  fold_slice_f32<UNROLL>(a, x, seg0, lane);
+}
+
+template <typename T, int UNROLL>
+__device__ __forceinline__ void fold_slice(WarpAcc& a, uint32_t (&w)[UNROLL][4], int seg0, int lane) {
+  if constexpr (sizeof(T) == 2) {
+    fold_slice_bf16<UNROLL>(a, w, seg0, lane);
+  } else {
+    float x[UNROLL][4];
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) x[j][c] = __uint_as_float(w[j][c]);
+    fold_slice_f32<UNROLL>(a, x, seg0, lane);
+  }
 }
 
 // Element-wise slice for rows without 16-byte structure and for the ragged
@@ -304,9 +311,11 @@ reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nse
   WarpAcc a;
   acc_init(a);
   constexpr int kSlice = UNROLL * 32;
+  constexpr uint32_t kFill = sizeof(T) == 2 ? kNegInf2 : 0xff800000u;
   for (int s0 = seg_begin + warp * kSlice; s0 < seg_end; s0 += kReduceWarps * kSlice) {
-    if constexpr (sizeof(T) == 2) warp_slice_bf16<UNROLL>(a, rv, s0, seg_end, lane);
-    else warp_slice_f32<UNROLL>(a, rv, s0, seg_end, lane);
+    uint32_t w[UNROLL][4];
+    load_slice<UNROLL>(w, rv, s0, seg_end, lane, kFill);
+    fold_slice<T, UNROLL>(a, w, s0, lane);
   }
   // ragged tail (fewer than kElems logits): last unit of the row, last warp
   if (split == splits - 1 && warp == kReduceWarps - 1 && nseg * kE < V)
