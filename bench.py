@@ -36,6 +36,10 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-reduction kernel, from the ncu
 # captures summarised under profiles/ (bytes); None where no capture exists.
 NCU_TRAFFIC_BYTES = {
+    "long_draft_batch": 282.8e6,                        # measured: 279.14 MB read + 3.67 MB written
+    "llama3_vocab_batch": 282.8e6 * 144 / 1088,         # the same kernel; traffic scales with the rows read
+    "high_batch_serving": 282.8e6 * (2304 * 152064) / (1088 * 128256),
+    "fused_lm_head": (1.0675e9 + 4.4e6) * 128256 / 64000,   # measured at V = 64000; scales with V
 }
 
 
@@ -407,7 +411,7 @@ def main():
     if w.hidden:
         run_fused(args, w)
         return
-    args.steps = args.steps or 20000
+    args.steps = args.steps or max(2000, int(0.6 / (w.rows * w.V * w.elem_bytes / 6.0e12)))   # ~0.6 s of timed work
     args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
 
     import torch

@@ -149,8 +149,9 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.  The load is
+// asynchronous: the registers are valid only after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -159,9 +160,10 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      : "r"(taddr)
+      : "memory");
 }
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -364,15 +366,21 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       tc_fence_after();
       const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + warp * 32;
       const int limit = p.V - v0;  // entries of this quarter that exist
+      // Two register sets: the tensor-memory load of block c+1 is in flight while block c is turned
+      // through shared memory and folded.
+      uint32_t ra[32], rb[32];
+      tmem_ld32_issue(tmem + lane_base, ra);
+      tmem_ld_wait();
+      if (nchunks == 1) {  // the tile's only block is in registers: hand the accumulators back to the MMA issuers
+        tc_fence_before();
+        mbar_arrive_remote(map_to_cta(tmem_empty, 0));
+      }
 #pragma unroll
       for (int c = 0; c < kChunks; ++c) {
         if (c < nchunks) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_base + (uint32_t)(c * kChunk), r);
-          if (c == nchunks - 1) {  // last read of this tile: hand the accumulators back to the MMA issuer
-            tc_fence_before();
-            mbar_arrive_remote(map_to_cta(tmem_empty, 0));
-          }
+          uint32_t (&r)[32] = (c & 1) ? rb : ra;
+          uint32_t (&rn)[32] = (c & 1) ? ra : rb;
+          if (c + 1 < nchunks) tmem_ld32_issue(tmem + lane_base + (uint32_t)((c + 1) * kChunk), rn);
           epi_bar();  // everyone is done reading the previous block
 #pragma unroll
           for (int i = 0; i < 32; ++i) turn[i * kTurnRow + warp * 32 + lane] = __uint_as_float(r[i]);
@@ -390,6 +398,13 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
               if (e >= limit) x[e] = kMaskFloor;
           }
           fold32(st[c], x, v0);
+          if (c + 1 < nchunks) {
+            tmem_ld_wait();
+            if (c + 2 == nchunks) {  // the tile's last block is in registers: hand the accumulators back
+              tc_fence_before();
+              mbar_arrive_remote(map_to_cta(tmem_empty, 0));
+            }
+          }
         }
       }
     }

@@ -16,6 +16,7 @@ tensors produced here, so both sides always see identical bits.
 from __future__ import annotations
 
 import hashlib
+import math
 from dataclasses import dataclass, replace
 from typing import Callable, Optional
 
@@ -66,7 +67,17 @@ FUSED = Workload("fused_lm_head", B=32, K=8, V=128256, dtype="bf16", scale=None,
                  spike_frac=0.0, spike=(0.0, 0.0), draft_mix=(0.7, 0.0, 0.3), steps=200,
                  hidden=8192)
 
-WORKLOADS = {w.name: w for w in (TINY, LLAMA3, LONG_DRAFT, SERVING, FUSED)}
+# The paper's own operating point (Section 3, implementation details): threshold 0.3 on the NORMALISED
+# entropy h = H / log|V| (= 3.53 nats at |V| = 128256), window W = 6, K = 15 drafts for the 70B target
+# and K = 25 for the 405B target, one sequence at a time.  Rows are drawn as for the Llama-3 batch.
+PAPER_70B = Workload("paper_default_70b", B=1, K=15, V=128256, dtype="bf16", scale=(0.5, 4.0),
+                     spike_frac=0.4, spike=(8.0, 16.0), draft_mix=(0.6, 0.3, 0.1), theta=0.3 * math.log(128256),
+                     W=6, steps=1000)
+PAPER_405B = Workload("paper_default_405b", B=1, K=25, V=128256, dtype="bf16", scale=(0.5, 4.0),
+                      spike_frac=0.4, spike=(8.0, 16.0), draft_mix=(0.6, 0.3, 0.1), theta=0.3 * math.log(128256),
+                      W=6, steps=1000)
+
+WORKLOADS = {w.name: w for w in (TINY, LLAMA3, LONG_DRAFT, SERVING, FUSED, PAPER_70B, PAPER_405B)}
 LONG_DRAFT_SETTINGS = [(th, W) for th in (0.5, 1.0, 2.0) for W in (1, 3, 5)]
 
 

@@ -252,3 +252,16 @@ def test_back_to_back_steps_with_stream_overlap():
     torch.cuda.synchronize()
     for (logits, draft), out in zip(steps, outs):
         assert_parity(out, oracle_step(logits, draft, 1.0, 3), "overlap")
+
+
+@pytest.mark.parametrize("name", ["paper_default_70b", "paper_default_405b"])
+@pytest.mark.parametrize("B", [1, 4, 16])
+def test_paper_default_operating_point(name, B):
+    # K = 15 / 25, W = 6, threshold 0.3 on the normalised entropy, small batches (few rows, many pieces per row)
+    w = S.shrink(S.WORKLOADS[name], B=B)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    logits, draft = draw(w, step=B)
+    check(fv, logits, draft, w.theta, w.W, what=f"{name} B={B} nats")
+    check(fv, logits, draft, 0.3, w.W, theta_unit="normalized", what=f"{name} B={B} normalized")
+    fv.set_stream_overlap(True)
+    check(fv, logits, draft, w.theta, w.W, what=f"{name} B={B} overlap")
