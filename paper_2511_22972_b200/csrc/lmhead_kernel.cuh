@@ -47,7 +47,6 @@
 #include <cuda.h>
 
 #include "fly_common.cuh"
-#include "mbarrier.cuh"
 
 namespace fly {
 namespace lmhead {
@@ -83,6 +82,7 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 static_assert(kMaxPos * 4 * 16 <= kStages * kBytesW, "final merge buffer reuses the weight ring");
 
 constexpr int kErrTimeoutProducer = 1, kErrTimeoutMma = 2, kErrTimeoutEpilogue = 3;
+constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;  // far above any legitimate wait (a tile takes ~50 us)
 
 struct Params {
   int R;          // positions handled by this launch (1..288)
@@ -97,6 +97,17 @@ struct Params {
 
 // ---- small PTX wrappers ------------------------------------------------------
 
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 // Arrives on a barrier of the CTA with rank `cta` in the pair (cluster-scope release).
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
@@ -116,6 +127,40 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Waits for the phase of `bar` with the given parity to complete.  Gives up when
+// the limit passes or when another role has already reported a failure.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63) == 0) {
+      if (*(volatile int*)status != 0) return false;
+      if (global_ns() - t0 > kWaitLimitNs) {
+        atomicCAS(status, 0, code);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
 // Tiled TMA load into THIS CTA's shared memory; the bytes are reported to `bar`, a shared::cluster
 // address that may lie in the other CTA of the pair.  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -149,9 +194,8 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.  The load is
-// asynchronous: the registers are valid only after tmem_ld_wait().
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
@@ -160,10 +204,9 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
         "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -366,21 +409,15 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       tc_fence_after();
       const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + warp * 32;
       const int limit = p.V - v0;  // entries of this quarter that exist
-      // Two register sets: the tensor-memory load of block c+1 is in flight while block c is turned
-      // through shared memory and folded.
-      uint32_t ra[32], rb[32];
-      tmem_ld32_issue(tmem + lane_base, ra);
-      tmem_ld_wait();
-      if (nchunks == 1) {  // the tile's only block is in registers: hand the accumulators back to the MMA issuers
-        tc_fence_before();
-        mbar_arrive_remote(map_to_cta(tmem_empty, 0));
-      }
 #pragma unroll
       for (int c = 0; c < kChunks; ++c) {
         if (c < nchunks) {
-          uint32_t (&r)[32] = (c & 1) ? rb : ra;
-          uint32_t (&rn)[32] = (c & 1) ? ra : rb;
-          if (c + 1 < nchunks) tmem_ld32_issue(tmem + lane_base + (uint32_t)((c + 1) * kChunk), rn);
+          uint32_t r[32];
+          tmem_ld32(tmem + lane_base + (uint32_t)(c * kChunk), r);
+          if (c == nchunks - 1) {  // last read of this tile: hand the accumulators back to the MMA issuer
+            tc_fence_before();
+            mbar_arrive_remote(map_to_cta(tmem_empty, 0));
+          }
           epi_bar();  // everyone is done reading the previous block
 #pragma unroll
           for (int i = 0; i < 32; ++i) turn[i * kTurnRow + warp * 32 + lane] = __uint_as_float(r[i]);
@@ -398,13 +435,6 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
               if (e >= limit) x[e] = kMaskFloor;
           }
           fold32(st[c], x, v0);
-          if (c + 1 < nchunks) {
-            tmem_ld_wait();
-            if (c + 2 == nchunks) {  // the tile's last block is in registers: hand the accumulators back
-              tc_fence_before();
-              mbar_arrive_remote(map_to_cta(tmem_empty, 0));
-            }
-          }
         }
       }
     }
