@@ -209,6 +209,11 @@ fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, in
  * pending, further fused steps give up early.  Logits-path kernels have no waits. */
 fly_status_t fly_verify_device_status(fly_verify_t* handle, void* cuda_stream);
 
+/* Self-test of that mechanism, safe to run anywhere: enqueues a one-thread kernel that waits, with a
+ * 2 ms limit, on a barrier nothing will complete.  The wait gives up, the kernel returns normally, and the
+ * next fly_verify_device_status reports FLY_ERR_TIMEOUT.  Nothing faults or hangs. */
+fly_status_t fly_verify_selftest_wait(fly_verify_t* handle, void* cuda_stream);
+
 /* Number of kernels the last fly_verify_run enqueued (for accounting). */
 int32_t fly_verify_last_launch_count(const fly_verify_t* handle);
 

@@ -21,7 +21,7 @@ FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
-    "fly_verify_device_status",
+    "fly_verify_device_status", "fly_verify_selftest_wait",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -77,6 +77,8 @@ def lib() -> C.CDLL:
     L.fly_verify_run_static.restype = C.c_int
     L.fly_verify_device_status.argtypes = [C.c_void_p, C.c_void_p]
     L.fly_verify_device_status.restype = C.c_int
+    L.fly_verify_selftest_wait.argtypes = [C.c_void_p, C.c_void_p]
+    L.fly_verify_selftest_wait.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -147,6 +149,10 @@ class FlyVerify:
     def device_status(self, stream: int = 0) -> int:
         """fly_verify_device_status: synchronises the stream; FLY_OK or FLY_ERR_TIMEOUT."""
         return int(lib().fly_verify_device_status(self._h, C.c_void_p(stream)))
+
+    def selftest_wait(self, stream: int = 0) -> int:
+        """fly_verify_selftest_wait: makes one bounded device-side wait run out on purpose (no fault)."""
+        return int(lib().fly_verify_selftest_wait(self._h, C.c_void_p(stream)))
 
     @property
     def last_launch_count(self) -> int:

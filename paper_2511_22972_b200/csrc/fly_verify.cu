@@ -427,6 +427,15 @@ fly_status_t fly_verify_device_status(fly_verify_t* h, void* cuda_stream) {
   return FLY_OK;
 }
 
+fly_status_t fly_verify_selftest_wait(fly_verify_t* h, void* cuda_stream) {
+  if (!h) return FLY_ERR_INVALID_ARG;
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  fly::lmhead::wait_selftest_kernel<<<1, 1, 0, static_cast<cudaStream_t>(cuda_stream)>>>(h->lm_status, 2000000ull);
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? FLY_OK : cuda_fail(h, e);
+}
+
 int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
 int32_t fly_verify_last_cuda_error(const fly_verify_t* h) { return h ? h->last_cuda_error : 0; }
 

@@ -47,6 +47,7 @@
 #include <cuda.h>
 
 #include "fly_common.cuh"
+#include "mbarrier.cuh"
 
 namespace fly {
 namespace lmhead {
@@ -82,7 +83,6 @@ static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 static_assert(kMaxPos * 4 * 16 <= kStages * kBytesW, "final merge buffer reuses the weight ring");
 
 constexpr int kErrTimeoutProducer = 1, kErrTimeoutMma = 2, kErrTimeoutEpilogue = 3;
-constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;  // far above any legitimate wait (a tile takes ~50 us)
 
 struct Params {
   int R;          // positions handled by this launch (1..288)
@@ -97,17 +97,6 @@ struct Params {
 
 // ---- small PTX wrappers ------------------------------------------------------
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
 // Arrives on a barrier of the CTA with rank `cta` in the pair (cluster-scope release).
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
@@ -127,40 +116,6 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Waits for the phase of `bar` with the given parity to complete.  Gives up when
-// the limit passes or when another role has already reported a failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  int spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 63) == 0) {
-      if (*(volatile int*)status != 0) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
-        atomicCAS(status, 0, code);
-        return false;
-      }
-    }
-  }
-  return true;
-}
-
 // Tiled TMA load into THIS CTA's shared memory; the bytes are reported to `bar`, a shared::cluster
 // address that may lie in the other CTA of the pair.  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -471,6 +426,17 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
+}
+
+// Exercises the bounded wait without any fault: one thread waits on a barrier that nothing will
+// ever complete; after limit_ns the wait gives up and records `code`.
+constexpr int kErrSelfTest = 9;
+__global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  const uint32_t b = smem_u32(&bar);
+  mbar_init(b, 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  mbar_wait(b, 0, status, kErrSelfTest, limit_ns);
 }
 
 }  // namespace lmhead

@@ -38,14 +38,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Waits for the phase of `bar` with the given parity to complete.  Gives up when
 // the limit passes or when another role has already reported a failure.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status, int code,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 63) == 0) {
       if (*(volatile int*)status != 0) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         atomicCAS(status, 0, code);
         return false;
       }

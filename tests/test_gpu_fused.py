@@ -170,3 +170,16 @@ def test_full_size_head_on_sampled_sequences():
         assert (toks[b, s[b]:] == -1).all()
         first_mismatch = next((i + 1 for i in range(K) if dr[b, i] != am[b, i]), K + 1)
         assert s[b] >= first_mismatch                              # s_FLy >= s_standard (Eq. 3 vs Eq. 11)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    # no fault, no hang: a one-thread kernel waits 2 ms on a barrier that nothing completes, gives up and
+    # records it; the host reads FLY_ERR_TIMEOUT once, and the next fused step is correct again
+    st = torch.cuda.current_stream().cuda_stream
+    fv = FlyVerify(4, 8, 2048, "bf16", hidden=256)
+    assert fv.device_status(st) == Bd.FLY_OK
+    assert fv.selftest_wait(st) == Bd.FLY_OK
+    assert fv.device_status(st) == Bd.FLY_ERR_TIMEOUT
+    assert fv.device_status(st) == Bd.FLY_OK                      # the record was cleared
+    fv.close()
+    run_and_check(4, 8, D=256, V=2048)

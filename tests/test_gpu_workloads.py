@@ -1,0 +1,70 @@
+"""The benchmark workloads at their FULL sizes, in the launch configuration bench.py times (consecutive
+steps overlapped, outputs of a step read back after later steps were enqueued), compared with the fp64
+oracle element by element.  The fused LM-head workload is in test_gpu_fused.py."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, synthetic as S, verify
+from tests._parity import assert_parity, draw, oracle_step
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def run_overlapped(fv, steps, theta, W, boundary="reject", chain=False):
+    """Enqueues all steps back to back on one stream, then compares every step with the oracle.
+    chain=True: one state buffer is carried from step to step (carry mode)."""
+    st = torch.cuda.current_stream().cuda_stream
+    fv.set_stream_overlap(True)
+    B, K1, _ = steps[0][0].shape
+    outs = [VerifyBuffers(B, K1 - 1, DEV) for _ in steps]
+    state = outs[0].state
+    snapshots = []
+    for (logits, draft), out in zip(steps, outs):
+        if chain:
+            out.state = state                        # every step reads and writes the same carried state
+        verify(fv, logits, draft, out, theta=theta, W=W, boundary=boundary, stream=st)
+        if chain:
+            snapshots.append(state.clone())          # stream-ordered copy of the state after this step
+    torch.cuda.synchronize()
+    assert fv.device_status(st) == 0
+    ref_state = np.array([[0, 0, -1]] * B) if chain else None
+    worst = 0.0
+    for n, ((logits, draft), out) in enumerate(zip(steps, outs)):
+        ref = oracle_step(logits, draft, theta, W, boundary, ref_state)
+        if chain:
+            out.state = snapshots[n]
+            ref_state = ref.state_out
+        worst = max(worst, assert_parity(out, ref, f"step {n}"))
+    return worst
+
+
+def test_tiny_verify_all_200_steps():
+    w = S.TINY
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype)
+    steps = [draw(w, step=s) for s in range(w.steps)]
+    assert run_overlapped(fv, steps, w.theta, w.W) <= 1e-4
+
+
+def test_llama3_vocab_batch_full_size():
+    w = S.LLAMA3
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype)
+    steps = [draw(w, step=s) for s in range(12)]
+    run_overlapped(fv, steps, w.theta, w.W)
+
+
+@pytest.mark.parametrize("setting", range(len(S.LONG_DRAFT_SETTINGS)))
+def test_long_draft_batch_full_size_every_setting(setting):
+    theta, W = S.LONG_DRAFT_SETTINGS[setting]
+    w = S.LONG_DRAFT
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype)
+    steps = [draw(w, step=s, setting=setting, thetas=[theta]) for s in range(2)]   # inputs regenerated per setting
+    run_overlapped(fv, steps, theta, W)
+
+
+def test_high_batch_serving_full_size_chained_rounds():
+    w = S.SERVING
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype)
+    steps = [draw(w, step=s) for s in range(6)]
+    run_overlapped(fv, steps, w.theta, w.W, boundary="carry", chain=True)
