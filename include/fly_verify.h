@@ -139,6 +139,35 @@ fly_status_t fly_verify_run(fly_verify_t* handle, const fly_verify_args_t* args,
  * remains a DEVICE pointer. */
 fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* args, void* cuda_stream);
 
+/* Vocabulary-parallel targets.  The paper runs its 405B target "distributed across four GPUs"
+ * (Section 3, implementation details); with a tensor-parallel LM head every GPU holds the logits of
+ * one slice of the vocabulary only.  Eq. 1 and Eq. 5 then split into a per-slice reduction and a
+ * merge: for a slice with maximum m_k, S_k = sum 2^(z - r_k) and u_k = sum 2^(z - r_k)(z - r_k)
+ * (z = logit * log2 e, r_k = m_k * log2 e), the whole row has m = max m_k,
+ * S = sum_k 2^(r_k - r) S_k, u = sum_k 2^(r_k - r)(u_k + (r_k - r) S_k), entropy
+ * H = ln2 (log2 S - u / S), and the greedy token is the index of the largest m_k (lowest index on
+ * ties).  One state per row and rank (16 bytes) is all that has to cross the interconnect.
+ *
+ * fly_verify_reduce_shard    on every rank: reduces this rank's logits [rows, vocab] (vocab = the
+ *                            handle's vocab = the slice width; row_stride elements between rows, 0 = vocab)
+ *                            to partial_out[rows].  vocab_offset = global id of the slice's first token.
+ * (all-gather partial_out over the ranks: [world, rows] states, e.g. with NCCL)
+ * fly_verify_run_partials    on every rank (or one): merges the gathered states and applies the gate and
+ *                            the deferred window exactly as fly_verify_run does.  args: as for
+ *                            fly_verify_run with logits, hidden and weight NULL; total_vocab = |V| (used for
+ *                            the draft-id range check and for a NORMALIZED threshold).
+ * All pointers dev.  Both calls are asynchronous on `cuda_stream` and allocate nothing. */
+typedef struct {
+  float max_logit;  /* m_k; a slice with no finite entry reports a value <= -999424 */
+  float sum_exp2;   /* S_k */
+  float sum_exp2_t; /* u_k */
+  int32_t argmax;   /* global token id of the first entry equal to m_k */
+} fly_partial_t;
+fly_status_t fly_verify_reduce_shard(fly_verify_t* handle, int32_t rows, const void* logits, int64_t row_stride,
+                                     int32_t vocab_offset, fly_partial_t* partial_out, void* cuda_stream);
+fly_status_t fly_verify_run_partials(fly_verify_t* handle, const fly_verify_args_t* args, const fly_partial_t* partials,
+                                     int32_t world, int32_t total_vocab, void* cuda_stream);
+
 /* The paper has no counterpart of this entry point; it exists for callers that
  * must not allocate device memory.
  *

@@ -21,7 +21,7 @@ FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
-    "fly_verify_device_status", "fly_verify_selftest_wait",
+    "fly_verify_device_status", "fly_verify_selftest_wait", "fly_verify_reduce_shard", "fly_verify_run_partials",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -79,6 +79,11 @@ def lib() -> C.CDLL:
     L.fly_verify_device_status.restype = C.c_int
     L.fly_verify_selftest_wait.argtypes = [C.c_void_p, C.c_void_p]
     L.fly_verify_selftest_wait.restype = C.c_int
+    L.fly_verify_reduce_shard.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
+    L.fly_verify_reduce_shard.restype = C.c_int
+    L.fly_verify_run_partials.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p, C.c_int32, C.c_int32,
+                                          C.c_void_p]
+    L.fly_verify_run_partials.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -149,6 +154,23 @@ class FlyVerify:
     def device_status(self, stream: int = 0) -> int:
         """fly_verify_device_status: synchronises the stream; FLY_OK or FLY_ERR_TIMEOUT."""
         return int(lib().fly_verify_device_status(self._h, C.c_void_p(stream)))
+
+    def reduce_shard(self, logits, vocab_offset: int, partial_out, stream: int = 0):
+        """fly_verify_reduce_shard: logits [rows, vocab_slice] (a strided view is fine) -> partial_out
+        [rows, 4] (any 16-byte element type, e.g. float32 x 4)."""
+        rows = logits.shape[0]
+        assert logits.shape[1] == self.vocab and logits.stride(1) == 1
+        st = lib().fly_verify_reduce_shard(self._h, int(rows), _ptr(logits), int(logits.stride(0)), int(vocab_offset),
+                                           _ptr(partial_out), C.c_void_p(stream))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_reduce_shard", lib().fly_verify_last_cuda_error(self._h))
+
+    def run_partials(self, args: fly_verify_args_t, partials, world: int, total_vocab: int, stream: int = 0):
+        """fly_verify_run_partials: partials [world, rows, 4] gathered from the ranks."""
+        st = lib().fly_verify_run_partials(self._h, C.byref(args), _ptr(partials), int(world), int(total_vocab),
+                                           C.c_void_p(stream))
+        if st != FLY_OK:
+            raise FlyError(st, "fly_verify_run_partials", lib().fly_verify_last_cuda_error(self._h))
 
     def selftest_wait(self, stream: int = 0) -> int:
         """fly_verify_selftest_wait: makes one bounded device-side wait run out on purpose (no fault)."""

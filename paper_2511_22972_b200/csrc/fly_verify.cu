@@ -55,7 +55,7 @@ struct fly_verify {
   int last_cuda_error = 0;
   // fused LM-head path (cfg.hidden > 0)
   fly::Partial* lm_partials = nullptr;  // [max_rows * sm_count]: one partial state per row and CTA
-  fly::Partial* lm_folded = nullptr;    // [max_rows]: the same, folded over the CTAs
+  fly::Partial* lm_folded = nullptr;    // [max_rows]: partial states folded over CTAs (fused path) or ranks
   int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
   int lm_pairs = 0;                     // CTA pairs that can be resident at once
   PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
@@ -249,7 +249,8 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     cudaLaunchAttribute attr[1];
     const unsigned warps = fly::kFoldThreads / 32;
     fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, true);
-    e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->lm_partials, grid, h->lm_folded, (int)rows);
+    e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->lm_partials, grid, (int64_t)grid,
+                           (int64_t)1, h->lm_folded, (int)rows, 0);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
   }
@@ -327,10 +328,14 @@ fly_status_t fly_verify_create(const fly_verify_config_t* c, fly_verify_t** out)
   if (e == cudaSuccess) e = cudaMemset(h->tickets, 0, (size_t)c->max_batch * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->lm_status, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(h->lm_status, 0, sizeof(int));
-  if (e != cudaSuccess) { cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_status); delete h; return FLY_ERR_CUDA; }
+  if (e == cudaSuccess) e = cudaMalloc(&h->lm_folded, (size_t)h->max_rows * sizeof(fly::Partial));
+  if (e != cudaSuccess) {
+    cudaFree(h->partials); cudaFree(h->tickets); cudaFree(h->lm_status); cudaFree(h->lm_folded);
+    delete h;
+    return FLY_ERR_CUDA;
+  }
   if (c->hidden > 0) {
     e = cudaMalloc(&h->lm_partials, (size_t)h->max_rows * h->sm_count * sizeof(fly::Partial));
-    if (e == cudaSuccess) e = cudaMalloc(&h->lm_folded, (size_t)h->max_rows * sizeof(fly::Partial));
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(fly::lmhead::lmhead_verify_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                fly::lmhead::kSmemBytes);
@@ -406,6 +411,68 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
       return FLY_OK;
   }
   return FLY_ERR_INVALID_ARG;
+}
+
+fly_status_t fly_verify_reduce_shard(fly_verify_t* h, int32_t rows, const void* logits, int64_t row_stride,
+                                     int32_t vocab_offset, fly_partial_t* partial_out, void* cuda_stream) {
+  if (!h || !logits || !partial_out) return FLY_ERR_INVALID_ARG;
+  if (rows < 1 || rows > h->max_rows || vocab_offset < 0) return FLY_ERR_INVALID_ARG;
+  const int V = h->cfg.vocab;
+  if (row_stride != 0 && row_stride < V) return FLY_ERR_INVALID_ARG;
+  if ((int64_t)vocab_offset + V > 0x7fffffff) return FLY_ERR_INVALID_ARG;
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t stride = row_stride ? row_stride : V;
+  fly::ScanParams none;
+  memset(&none, 0, sizeof(none));  // tickets == NULL: no acceptance scan in this launch
+  int splits = 1;
+  cudaError_t e;
+  if (h->cfg.logits_dtype == FLY_BF16)
+    e = launch_reduce<__nv_bfloat16>(h, logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, none, false);
+  else
+    e = launch_reduce<float>(h, logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, none, false);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  const unsigned warps = fly::kFoldThreads / 32;
+  fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, true);
+  e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->partials, splits, (int64_t)splits, (int64_t)1,
+                         reinterpret_cast<fly::Partial*>(partial_out), (int)rows, (int)vocab_offset);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->last_launches = 2;
+  return FLY_OK;
+}
+
+fly_status_t fly_verify_run_partials(fly_verify_t* h, const fly_verify_args_t* a, const fly_partial_t* partials,
+                                     int32_t world, int32_t total_vocab, void* cuda_stream) {
+  if (!h || !a || !partials || world < 1 || world > 1024 || total_vocab < 1) return FLY_ERR_INVALID_ARG;
+  if (a->logits || a->hidden || a->weight) return FLY_ERR_INVALID_ARG;  // the logits were reduced by the shards
+  fly_verify_args_t chk = *a;
+  chk.logits = partials;  // satisfies the "exactly one input" rule of the common checks
+  fly_status_t s = check_args(h, &chk);
+  if (s != FLY_OK) return s;
+  DeviceGuard g(h->cfg.device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t rows = (int64_t)a->B * (a->K + 1);
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  const unsigned warps = fly::kFoldThreads / 32;
+  fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, false);
+  // all-gather layout: [world, rows]
+  cudaError_t e = cudaLaunchKernelEx(&cfg, fly::fold_partials, reinterpret_cast<const fly::Partial*>(partials), (int)world,
+                                     (int64_t)1, (int64_t)rows, h->lm_folded, (int)rows, 0);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  fly::ScanParams sp = scan_params(h, a, h->lm_folded, 1);
+  sp.V = total_vocab;
+  double th = a->theta;
+  if (a->theta_unit == FLY_THETA_NORMALIZED) th *= std::log((double)total_vocab);
+  sp.theta_nats = (float)th;
+  e = launch_scan(sp, st);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->last_launches = 2;
+  return FLY_OK;
 }
 
 fly_status_t fly_verify_device_status(fly_verify_t* h, void* cuda_stream) {

@@ -159,23 +159,27 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
   }
 }
 
-// Folds the n partial states of every row into one (out[row]); one warp per row.  The fused LM-head
-// kernel leaves one partial state per row and CTA; folding them with 32 lanes in parallel keeps the
-// acceptance scan's per-lane loop short.
+// Folds the n partial states of every row into one (out[row]); one warp per row.  Part j of row r
+// is in[r * row_stride + j * part_stride].  The fused LM-head kernel leaves one partial state per row
+// and CTA, a vocabulary-parallel target one per row and rank; folding them with 32 lanes in parallel
+// keeps the acceptance scan's per-lane loop short.  idx_offset is added to the winning index (a
+// vocabulary shard reports global token ids).
 constexpr int kFoldThreads = 128;
-__global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __restrict__ in, int n,
-                                                              Partial* __restrict__ out, int rows) {
+__global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __restrict__ in, int n, int64_t row_stride,
+                                                              int64_t part_stride, Partial* __restrict__ out, int rows,
+                                                              int idx_offset) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kFoldThreads / 32) + (threadIdx.x >> 5);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the producer grid has completed
   asm volatile("griddepcontrol.launch_dependents;");
   if (row >= rows) return;
-  const Partial* src = in + (int64_t)row * n;
+  const Partial* src = in + (int64_t)row * row_stride;
   Partial acc = empty_partial();
   for (int j0 = 0; j0 < n; j0 += 128) {  // four independent loads in flight per lane
     Partial q[4];
 #pragma unroll
-    for (int t = 0; t < 4; ++t) q[t] = (j0 + t * 32 + lane < n) ? ld_partial_cg(src + j0 + t * 32 + lane) : empty_partial();
+    for (int t = 0; t < 4; ++t)
+      q[t] = (j0 + t * 32 + lane < n) ? ld_partial_cg(src + (int64_t)(j0 + t * 32 + lane) * part_stride) : empty_partial();
 #pragma unroll
     for (int t = 0; t < 4; ++t) merge_partial(acc, q[t]);
   }
@@ -184,7 +188,10 @@ __global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __r
     const Partial q = shfl_xor_partial(acc, o);
     merge_partial(acc, q);
   }
-  if (lane == 0) out[row] = acc;
+  if (lane == 0) {
+    if (acc.idx != kIdxNone) acc.idx += idx_offset;
+    out[row] = acc;
+  }
 }
 
 // Stand-alone launch: one warp per sequence, after the row reduction.

@@ -77,6 +77,26 @@ def shard_sequences(total_B: int, r: Ranks) -> range:
     return range(lo, lo + per + (1 if r.rank < extra else 0))
 
 
+def shard_vocab(V: int, r: Ranks, align: int = 8):
+    """(offset, width) of this rank's slice of the vocabulary; slice starts are multiples of `align`
+    tokens so that every slice keeps 16-byte structure."""
+    per = -(-V // r.world)
+    per = -(-per // align) * align
+    lo = min(V, r.rank * per)
+    return lo, min(V, lo + per) - lo
+
+
+def all_gather_partials(r: Ranks, partial: torch.Tensor) -> torch.Tensor:
+    """All-gathers the per-row partial states of a vocabulary-parallel step: [rows, 4] on every rank ->
+    [world, rows, 4] on every rank (16 bytes per row and rank: latency-bound, one NCCL call)."""
+    if r.world == 1:
+        return partial.unsqueeze(0)
+    import torch.distributed as dist
+    out = torch.empty((r.world,) + tuple(partial.shape), dtype=partial.dtype, device=partial.device)
+    dist.all_gather(list(out.unbind(0)), partial.contiguous())   # one slot of `out` per rank, in rank order
+    return out
+
+
 def finalize(r: Ranks) -> None:
     if r.world > 1:
         import torch.distributed as dist

@@ -17,9 +17,16 @@ WORKER = textwrap.dedent("""
     shard = D.shard_sequences(37, r)
     slow = D.max_over_ranks(r, 10.0 + 5.0 * r.rank)
     total = D.sum_over_ranks(r, len(shard))
+    # vocabulary-parallel plumbing: slice of the vocabulary, all-gather of the per-row partial states
+    import torch
+    off, width = D.shard_vocab(128256, r)
+    mine = torch.full((5, 4), float(r.rank + 1))
+    mine[:, 3] = off
+    gathered = D.all_gather_partials(r, mine)
     D.barrier(r)
     print(json.dumps({"rank": r.rank, "world": r.world, "lo": shard.start, "hi": shard.stop,
-                      "slow": slow, "total": total, "main": r.is_main}))
+                      "slow": slow, "total": total, "main": r.is_main, "voff": off, "vwidth": width,
+                      "gshape": list(gathered.shape), "g0": gathered[0, 0].tolist(), "g1": gathered[1, 4].tolist()}))
     D.finalize(r)
 """) % ROOT
 
@@ -52,6 +59,9 @@ def test_two_gloo_ranks_shard_and_reduce():
     assert all(d["slow"] == 15.0 for d in outs)         # max over ranks, seen by every rank
     assert all(d["total"] == 37.0 for d in outs)
     assert outs[0]["main"] and not outs[1]["main"]
+    assert [(d["voff"], d["vwidth"]) for d in outs] == [(0, 64128), (64128, 64128)]
+    for d in outs:                                      # every rank holds every rank's states, in rank order
+        assert d["gshape"] == [2, 5, 4] and d["g0"] == [1.0, 1.0, 1.0, 0.0] and d["g1"] == [2.0, 2.0, 2.0, 64128.0]
 
 
 def test_single_rank_needs_no_process_group():
@@ -61,6 +71,8 @@ def test_single_rank_needs_no_process_group():
         r = D.init_from_env("nccl")
         assert (r.rank, r.world, r.backend) == (0, 1, "")
         assert D.max_over_ranks(r, 3.5) == 3.5 and list(D.shard_sequences(5, r)) == [0, 1, 2, 3, 4]
+        assert D.shard_vocab(50257, r) == (0, 50257)
+        assert [D.shard_vocab(50257, D.Ranks(k, 7, 0, "")) for k in (0, 6)] == [(0, 7184), (43104, 7153)]
         D.barrier(r)
         D.finalize(r)
     finally:
