@@ -122,7 +122,15 @@ typedef struct {
   int32_t* target_argmax; /* dev [B, K+1] or NULL: y_i of Eq. 1, lowest index among equal maxima */
   float* entropy;         /* dev [B, K+1] or NULL: H_i in nats (numerator of Eq. 5) */
   uint32_t* row_flags;    /* dev [B, K+1] or NULL: bit 0 non-finite logit (NaN, +inf, or no finite entry);
-                             bit 1 draft id outside [0, V) (treated as a mismatch) */
+                             bit 1 draft id outside [0, V) (treated as a mismatch);
+                             bit 2 caller-supplied target token outside [0, V) (mismatch, never deferred) */
+
+  /* Optional (NULL = greedy): dev [B, K+1] tokens y_1..y_{K+1} that the caller drew from the target
+   * distributions, e.g. by sampling at temperature 1.  The paper's method text defines y_i only as the
+   * argmax (Eq. 1) although it reports temperature-1 results, so this is a hook, not the paper's rule:
+   * the given tokens replace the argmax in the match indicator (Eq. 2) and in the emitted tokens;
+   * the entropy gate still uses the entropy of the logits.  target_argmax still reports the argmax. */
+  const int32_t* target_tokens;
 } fly_verify_args_t;
 
 /* Runs one verification step on `cuda_stream` (a cudaStream_t; NULL = default

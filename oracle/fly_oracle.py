@@ -33,6 +33,7 @@ import numpy as np
 
 FLAG_NONFINITE = 1  # a NaN or +inf logit, or a row with no finite logit
 FLAG_BAD_DRAFT = 2  # a draft token id outside [0, V)
+FLAG_BAD_TARGET = 4  # a caller-supplied target token outside [0, V)
 
 
 def row_stats(x: np.ndarray):
@@ -305,11 +306,17 @@ class BatchResult(NamedTuple):
 
 def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
                  theta_unit: str = "nats", boundary: str = "reject",
-                 state_in: Optional[np.ndarray] = None) -> BatchResult:
+                 state_in: Optional[np.ndarray] = None,
+                 target_tokens: Optional[np.ndarray] = None) -> BatchResult:
     """One verification step.  logits [B, K+1, V] float64 (exactly widened
     input bits), draft [B, K] integer.  Entropy is computed for every row
     (the paper needs it only at mismatches; the extra rows change nothing).
-    A draft id outside [0, V) counts as a mismatch and is flagged."""
+    A draft id outside [0, V) counts as a mismatch and is flagged.
+
+    target_tokens [B, K+1] (optional, an extension outside the paper's method text, which defines y_i
+    only as the argmax of Eq. 1): tokens the caller drew from the target distributions.  They take the
+    place of y_i in Eq. 2 and in the emitted tokens; the gate still uses the entropy of the logits and
+    target_argmax still reports the argmax.  An id outside [0, V) is flagged and never accepted."""
     logits = np.asarray(logits, dtype=np.float64)
     B, K1, V = logits.shape
     K = K1 - 1
@@ -323,11 +330,23 @@ def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
     rb = np.zeros(B, dtype=np.int32)
     toks = np.full((B, K1), -1, dtype=np.int32)
     st_out = np.zeros((B, 3), dtype=np.int32)
+    y_used = y.copy()
+    if target_tokens is not None:
+        tt = np.asarray(target_tokens).reshape(B, K1)
+        for b in range(B):
+            for i in range(K1):
+                if flags[b, i] & FLAG_NONFINITE:
+                    continue                      # the row is unusable whatever the caller drew
+                if 0 <= int(tt[b, i]) < V:
+                    y_used[b, i] = int(tt[b, i])
+                else:
+                    flags[b, i] |= FLAG_BAD_TARGET
+                    y_used[b, i] = 0
     for b in range(B):
         for i in range(K):
             if not (0 <= int(draft[b, i]) < V):
                 flags[b, i] |= FLAG_BAD_DRAFT
-        delta = match_indicator(draft[b], y[b, :K])
+        delta = match_indicator(draft[b], y_used[b, :K])
         # The paper does not treat invalid input.  Reading used by both sides: a
         # flagged position counts as a mismatch that the gate never defers, so
         # an invalid token id can never be emitted.
@@ -336,10 +355,10 @@ def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
             if flags[b, i]:
                 delta[i] = 0
         if boundary == "reject":
-            res = verify_round_paper(delta, Hg, th, W, draft[b], y[b])
+            res = verify_round_paper(delta, Hg, th, W, draft[b], y_used[b])
         elif boundary == "carry":
             sin = ZERO_STATE if state_in is None else State(*[int(t) for t in state_in[b]])
-            res = verify_round_carry(delta, Hg, th, W, draft[b], y[b], sin)
+            res = verify_round_carry(delta, Hg, th, W, draft[b], y_used[b], sin)
         else:
             raise ValueError(boundary)
         acc[b] = res.accept_len

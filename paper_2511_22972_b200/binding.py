@@ -42,6 +42,7 @@ class fly_verify_args_t(C.Structure):
         ("state_in", C.c_void_p), ("state_out", C.c_void_p),
         ("accept_len", C.c_void_p), ("rollback", C.c_void_p), ("out_tokens", C.c_void_p),
         ("target_argmax", C.c_void_p), ("entropy", C.c_void_p), ("row_flags", C.c_void_p),
+        ("target_tokens", C.c_void_p),
     ]
 
 
@@ -182,7 +183,8 @@ class FlyVerify:
 
     def make_args(self, B, K, draft, accept_len, out_tokens, logits=None, row_stride=0, hidden=None,
                   weight=None, theta=1.0, theta_unit="nats", W=3, boundary="reject", state_in=None,
-                  state_out=None, rollback=None, target_argmax=None, entropy=None, row_flags=None):
+                  state_out=None, rollback=None, target_argmax=None, entropy=None, row_flags=None,
+                  target_tokens=None):
         a = fly_verify_args_t()
         a.B, a.K = int(B), int(K)
         a.logits, a.row_stride = _ptr(logits), int(row_stride)
@@ -195,6 +197,7 @@ class FlyVerify:
         a.state_in, a.state_out = _ptr(state_in), _ptr(state_out)
         a.accept_len, a.rollback, a.out_tokens = _ptr(accept_len), _ptr(rollback), _ptr(out_tokens)
         a.target_argmax, a.entropy, a.row_flags = _ptr(target_argmax), _ptr(entropy), _ptr(row_flags)
+        a.target_tokens = _ptr(target_tokens)
         return a
 
     def run(self, args: fly_verify_args_t, stream: int = 0):

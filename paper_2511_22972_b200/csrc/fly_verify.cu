@@ -68,7 +68,7 @@ struct fly_verify {
   // staging for fly_verify_run_host (allocated on first use)
   void* st_logits = nullptr;
   size_t st_logits_bytes = 0;
-  int32_t* st_ints = nullptr;  // draft | state_in | state_out | accept | rollback | tokens | argmax | flags
+  int32_t* st_ints = nullptr;  // draft | state_in | state_out | accept | rollback | tokens | argmax | flags | target tokens
   float* st_entropy = nullptr;
 };
 
@@ -284,6 +284,7 @@ fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, con
   p.target_argmax = a->target_argmax;
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
+  p.target_tokens = a->target_tokens;
   return p;
 }
 
@@ -535,6 +536,7 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   p.target_argmax = a->target_argmax;
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
+  p.target_tokens = a->target_tokens;
 
   const bool fused_tail = h->scan_mode == 0;
   cudaError_t e;
@@ -576,7 +578,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
   if (!h->st_ints) {
     // staging sized once for the largest run this handle allows
     const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
-    const size_t ints = (size_t)(mb * (mk1 - 1) + 3 * mb + 3 * mb + mb + mb + 3 * mb * mk1);
+    const size_t ints = (size_t)(mb * (mk1 - 1) + 3 * mb + 3 * mb + mb + mb + 4 * mb * mk1);
     if ((e = cudaMalloc(&h->st_ints, ints * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
     if ((e = cudaMalloc(&h->st_entropy, (size_t)(mb * mk1) * sizeof(float))) != cudaSuccess) return cuda_fail(h, e);
   }
@@ -605,6 +607,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
   int32_t* d_tokens = d_rollback + mb;
   int32_t* d_argmax = d_tokens + mb * mk1;
   int32_t* d_flags = d_argmax + mb * mk1;
+  int32_t* d_target = d_flags + mb * mk1;
 
   if (a->logits && (e = cudaMemcpyAsync(h->st_logits, a->logits, logit_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
@@ -614,6 +617,9 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     return cuda_fail(h, e);
   if (a->state_in &&
       (e = cudaMemcpyAsync(d_state_in, a->state_in, (size_t)B * 12, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return cuda_fail(h, e);
+  if (a->target_tokens &&
+      (e = cudaMemcpyAsync(d_target, a->target_tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
 
   fly_verify_args_t d = *a;
@@ -628,6 +634,7 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
   d.target_argmax = a->target_argmax ? d_argmax : nullptr;
   d.entropy = a->entropy ? h->st_entropy : nullptr;
   d.row_flags = a->row_flags ? reinterpret_cast<uint32_t*>(d_flags) : nullptr;
+  d.target_tokens = a->target_tokens ? d_target : nullptr;
   s = fly_verify_run(h, &d, cuda_stream);
   if (s != FLY_OK) return s;
 
@@ -734,6 +741,7 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
   p.target_argmax = a->target_argmax;
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
+  p.target_tokens = a->target_tokens;
 
   // The arrival counters must start at zero, whatever an earlier call left behind.
   cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4, st);

@@ -35,6 +35,7 @@ struct ScanParams {
   int32_t* target_argmax;   // [B, K+1] or null
   float* entropy;           // [B, K+1] or null
   uint32_t* row_flags;      // [B, K+1] or null
+  const int32_t* target_tokens;  // [B, K+1] or null: the caller's y_i instead of the argmax
 };
 
 struct RoundOutcome {
@@ -110,6 +111,11 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
       if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx <= kMaskFloor) flag |= kFlagNonFinite;
       int y = acc.idx;
       if (flag || y < 0 || y >= p.V) y = 0;  // keep every emitted id in range
+      const int greedy = y;
+      if (p.target_tokens && !(flag & kFlagNonFinite)) {  // the caller drew y_i itself
+        y = p.target_tokens[row];
+        if (y < 0 || y >= p.V) { flag |= kFlagBadTarget; y = 0; }
+      }
       sm_y[i] = y;
       if (i < K) {
         const int d = p.draft[(int64_t)b * K + i];
@@ -117,7 +123,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
         is_mism = (d != y) || flag;
         is_defer = (H >= p.theta_nats) && !flag;  // a flagged position is never kept
       }
-      if (p.target_argmax) p.target_argmax[row] = y;
+      if (p.target_argmax) p.target_argmax[row] = greedy;
       if (p.entropy) p.entropy[row] = H;
       if (p.row_flags) p.row_flags[row] = flag;
     }

@@ -265,3 +265,36 @@ def test_paper_default_operating_point(name, B):
     check(fv, logits, draft, 0.3, w.W, theta_unit="normalized", what=f"{name} B={B} normalized")
     fv.set_stream_overlap(True)
     check(fv, logits, draft, w.theta, w.W, what=f"{name} B={B} overlap")
+
+
+def test_caller_supplied_target_tokens():
+    # the hook for sampled (temperature-1) target tokens: they replace the argmax in Eq. 2 and in the output
+    from paper_2511_22972_b200 import VerifyBuffers
+    w = small("bf16", B=12, K=8, V=32064)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    logits, draft = draw(w, step=21)
+    g = torch.Generator().manual_seed(3)
+    y = logits.float().argmax(dim=2).to(torch.int32).cpu()
+    tt = y.clone()
+    resample = torch.rand(tt.shape, generator=g) < 0.3
+    tt[resample] = torch.randint(0, w.V, (int(resample.sum()),), generator=g, dtype=torch.int32)
+    agree = torch.rand(w.B, w.K, generator=g) < 0.3           # the sample sometimes agrees with the draft
+    tt[:, :w.K][agree] = draft.cpu()[agree]
+    tt[3, 2] = w.V                                            # out of range: flagged, never accepted
+    tt[5, w.K] = -2
+    tt = tt.to(DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    for boundary, state in (("reject", None), ("carry", [[1, 2, 5]] * w.B)):
+        out = VerifyBuffers(w.B, w.K, DEV)
+        if state is not None:
+            out.state.copy_(torch.as_tensor(state, dtype=torch.int32))
+        a = fv.make_args(w.B, w.K, draft, out.accept_len, out.out_tokens, logits=logits, theta=1.0, W=3,
+                         boundary=boundary, state_in=out.state if state is not None else None, state_out=out.state,
+                         rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
+                         row_flags=out.row_flags, target_tokens=tt)
+        fv.run(a, st)
+        torch.cuda.synchronize()
+        ref = O.verify_batch(logits.double().cpu().numpy(), draft.cpu().numpy(), 1.0, 3, boundary=boundary,
+                             state_in=None if state is None else np.asarray(state), target_tokens=tt.cpu().numpy())
+        assert ref.row_flags[3, 2] == 4 and ref.row_flags[5, w.K] == 4
+        assert_parity(out, ref, f"target tokens {boundary}")

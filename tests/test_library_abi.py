@@ -41,7 +41,7 @@ def test_struct_layout_matches_the_header():
     a = Bd.fly_verify_args_t
     assert a.logits.offset == 8 and a.row_stride.offset == 16 and a.draft.offset == 40
     assert a.theta.offset == 48 and a.theta_unit.offset == 56 and a.W.offset == 60 and a.boundary.offset == 64
-    assert a.state_in.offset == 72 and a.row_flags.offset == 128 and C.sizeof(a) == 136
+    assert a.state_in.offset == 72 and a.row_flags.offset == 128 and a.target_tokens.offset == 136 and C.sizeof(a) == 144
 
 
 @pytest.mark.parametrize("cfg", [

@@ -170,3 +170,28 @@ def test_verify_batch_end_to_end_tiny():
     bad = draft.copy(); bad[1, 0] = 4
     r3 = O.verify_batch(logits, bad, theta=1.0, W=W)
     assert r3.accept_len[1] == 1 and r3.row_flags[1, 0] == O.FLAG_BAD_DRAFT
+
+
+def test_caller_supplied_target_tokens_replace_the_argmax_in_eq2_and_in_the_output():
+    # extension outside the paper's text (which defines y_i as the argmax only)
+    import numpy as np
+    from oracle import fly_oracle as O
+    rng = np.random.default_rng(0)
+    B, K, V = 3, 5, 11
+    logits = rng.normal(size=(B, K + 1, V)) * 3
+    y = logits.argmax(axis=2)
+    draft = y[:, :K].copy()
+    draft[0, 2] = (draft[0, 2] + 1) % V                    # one mismatch against the argmax
+    base = O.verify_batch(logits, draft, theta=1e9, W=2)    # exact-match acceptance
+    same = O.verify_batch(logits, draft, theta=1e9, W=2, target_tokens=y)
+    assert np.array_equal(base.accept_len, same.accept_len) and np.array_equal(base.out_tokens, same.out_tokens)
+    assert base.accept_len[0] == 3
+    tt = y.copy()
+    tt[0, 2] = draft[0, 2]                                 # the caller's sample agrees with the draft there ...
+    tt[1, 0] = (y[1, 0] + 3) % V                           # ... and disagrees with a draft that matched the argmax
+    tt[2, K] = V + 4                                       # bonus token out of range
+    got = O.verify_batch(logits, draft, theta=1e9, W=2, target_tokens=tt)
+    assert got.accept_len.tolist() == [K + 1, 1, K + 1]
+    assert got.out_tokens[1, 0] == tt[1, 0] and got.out_tokens[0, K] == y[0, K]
+    assert got.row_flags[2, K] == O.FLAG_BAD_TARGET and got.out_tokens[2, K] == 0
+    assert np.array_equal(got.target_argmax, y)            # the argmax is still reported as such
