@@ -23,22 +23,23 @@
 // weights (the only large operand) stream from HBM exactly once.
 //
 // Pairs are persistent: pair i walks vocabulary tiles i, i + #pairs, ...  Warp
-// roles in each CTA: 0-3 epilogue (they own the four 32-lane quarters of tensor
-// memory), 4 weight producer, 5 hidden producer, 6 and 7 MMA issuers (leader CTA
-// only; one per accumulator).
+// roles in each CTA: 0-7 epilogue (two groups of four; warp w reads the 32-lane
+// quarter w % 4 of tensor memory), 8 weight producer, 9 hidden producer, 10 and
+// 11 MMA issuers (leader CTA only; one per accumulator).
 // "Full" barriers live in the leader: both CTAs' TMA loads report their bytes
 // there.  The leader's tcgen05.commit releases a stage in both CTAs.
 //
 // Epilogue.  A thread that reads tensor memory owns one vocabulary entry and
 // sees all positions; the reduction runs over the vocabulary.  The tile is
-// therefore turned through shared memory 32 positions at a time: the four
-// epilogue warps store their 32 x 32 block transposed, then thread
-// (position i, vocabulary quarter q) streams the 32 logits of its quarter and
+// therefore turned through shared memory 16 positions at a time (the two
+// epilogue groups take alternate blocks, each with a buffer of its own): the
+// group's four warps store their 32 x 16 blocks transposed, then thread
+// (position i, vocabulary eighth e) streams the 16 logits of its eighth and
 // folds them into a running (max, sum 2^t, sum 2^t t, argmax) held in registers
 // for the whole kernel - the same state and the same arithmetic as the row
 // reduction of the logits path, with no cross-lane traffic.  At the end the
-// four quarters are merged and the CTA writes one Partial per position; the
-// acceptance scan folds the gridDim.x partials of every row.
+// eight eighths are merged and the CTA writes one Partial per position; a
+// later kernel folds the gridDim.x partials of every row.
 //
 // Every wait on a barrier is bounded: a wait that runs out records a code in
 // *status, and all roles fall through to the common exit (tensor memory is
@@ -64,12 +65,16 @@ constexpr int kBytesWBox = kBlockK * 64 * 2;        // one TMA box: 64 entries x
 constexpr int kBoxPos = kHalfN / 2;                 // positions per TMA box: this CTA's half of one accumulator
 constexpr int kBytesHHalf = kBoxPos * kBlockK * 2;  // 9 KB
 constexpr int kBytesH = 2 * kBytesHHalf;            // both accumulators
-constexpr int kChunk = 32;                          // positions turned through shared memory at a time
-constexpr int kChunks = kMaxPos / kChunk;           // 9
+constexpr int kChunk = 16;                          // positions turned through shared memory at a time
+constexpr int kChunks = kMaxPos / kChunk;           // 18 per tile, dealt alternately to the two epilogue groups
+constexpr int kGroupChunks = kChunks / 2;           // 9 per group: the running states one thread holds
 constexpr int kTurnRow = kBlockV + 4;               // words per position row (+4: conflict-free 128-bit reads)
-constexpr int kTurnBytes = kChunk * kTurnRow * 4;
-constexpr int kEpiThreads = 128;
-constexpr int kThreads = 256;
+constexpr int kTurnGroupBytes = kChunk * kTurnRow * 4;
+constexpr int kTurnBytes = 2 * kTurnGroupBytes;     // one turning buffer per epilogue group
+constexpr int kEpiWarps = 8;                        // two groups of four warps (a warp reads tensor-memory lanes 32*(warp%4)..)
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kWarpW = kEpiWarps, kWarpH = kEpiWarps + 1, kWarpMma = kEpiWarps + 2;  // producers, MMA issuers
+constexpr int kThreads = (kEpiWarps + 4) * 32;
 constexpr int kTmemCols = 512;
 
 constexpr int kOffW = 0;
@@ -80,7 +85,7 @@ constexpr int kNumBars = 2 * kStages + 2;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;
 constexpr int kSmemBytes = kOffMisc + 32 + 1024;    // + slack to align the base to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
-static_assert(kMaxPos * 4 * 16 <= kStages * kBytesW, "final merge buffer reuses the weight ring");
+static_assert(kMaxPos * 8 * 16 <= kStages * kBytesW, "final merge buffer reuses the weight ring");
 
 constexpr int kErrTimeoutProducer = 1, kErrTimeoutMma = 2, kErrTimeoutEpilogue = 3;
 
@@ -149,21 +154,20 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// 32 lanes x 32 columns of fp32: thread = lane, register i = column col0 + i.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 lanes x 16 columns of fp32: thread = lane, register i = column col0 + i.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr));
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Named barriers: 1 and 2 for the two epilogue groups (128 threads each), 3 for all epilogue threads.
+__device__ __forceinline__ void group_bar(int group) { asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory"); }
+__device__ __forceinline__ void epi_all_bar() { asm volatile("bar.sync 3, 256;" ::: "memory"); }
 
 // ---- descriptors ---------------------------------------------------------------
 // Shared-memory matrix descriptor of tcgen05.mma (64 bits).  Low word: start address and leading
@@ -186,11 +190,11 @@ struct Stream {
   int idx;
 };
 
-// Folds 32 consecutive vocabulary entries x[0..31] (the first one has index v0) into st.
-__device__ __forceinline__ void fold32(Stream& st, float (&x)[32], int v0) {
+// Folds 16 consecutive vocabulary entries x[0..15] (the first one has index v0) into st.
+__device__ __forceinline__ void fold16(Stream& st, float (&x)[16], int v0) {
   float lm = kMaskFloor;
 #pragma unroll
-  for (int e = 0; e < 32; ++e) {
+  for (int e = 0; e < 16; ++e) {
     x[e] = max_nan_f32(x[e], kMaskFloor);  // masked entries stay finite; NaN survives and ends in S
     lm = fmaxf(lm, x[e]);
   }
@@ -200,16 +204,16 @@ __device__ __forceinline__ void fold32(Stream& st, float (&x)[32], int v0) {
     st.u = sc * fmaf(d, st.S, st.u);
     st.S *= sc;
     st.mx = lm;
-    int first = 31;
+    int first = 15;
 #pragma unroll
-    for (int e = 31; e >= 0; --e)
+    for (int e = 15; e >= 0; --e)
       if (x[e] == lm) first = e;
     st.idx = v0 + first;
   }
   const float nr = -st.mx * kLog2e;
   float S0 = 0.f, S1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
-  for (int e = 0; e < 32; e += 2) {
+  for (int e = 0; e < 16; e += 2) {
     const float t0 = fmaf(x[e], kLog2e, nr), t1 = fmaf(x[e + 1], kLog2e, nr);
     const float e0 = ex2_approx(t0), e1 = ex2_approx(t1);
     S0 += e0;
@@ -236,7 +240,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   auto empty = [&](int s) { return bar0 + 8u * (kStages + s); };
   const uint32_t tmem_full = bar0 + 8u * (2 * kStages);
   const uint32_t tmem_empty = tmem_full + 8u;
-  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1] epilogue go flag
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1], [2] go flags of the epilogue groups
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();  // 0: leader of the pair (issues the MMAs, owns the "full" barriers)
@@ -263,7 +267,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
 
   const int my_tiles = pair < p.num_tiles ? (p.num_tiles - 1 - pair) / npairs + 1 : 0;
 
-  if (warp == 4) {
+  if (warp == kWarpW) {
     // ---------------- weight producer: this CTA's 128 vocabulary entries ----------------
     if (lane == 0) {
       int issued = 0;
@@ -282,7 +286,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == kWarpH) {
     // ---------------- hidden-state producer: this CTA's half of each accumulator's positions ----------------
     if (lane == 0) {
       int issued = 0;
@@ -303,11 +307,11 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
         }
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= kWarpMma) {
     // ---------------- MMA issuers (leader CTA): warp 6 feeds accumulator 0, warp 7 accumulator 1 ----------------
     // One thread cannot issue MMAs, commits and barrier waits fast enough to keep the tensor pipe
     // busy with two 144-column MMAs per 16 hidden dims, so each accumulator has an issuer of its own.
-    const int half = warp - 6;
+    const int half = warp - kWarpMma;
     if (lane == 0 && rank == 0 && (half == 0 || p.n1 > 0)) {
       const uint32_t idesc = instr_desc(half == 0 ? p.n0 : p.n1);
       const uint32_t d_tmem = tmem + (uint32_t)(half * kHalfN);
@@ -349,66 +353,77 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       }
     }
   } else {
-    // ---------------- epilogue: warps 0..3, thread = (position lane, vocabulary quarter warp) ----------------
-    Stream st[kChunks];
+    // ---------------- epilogue: warps 0..7 = two groups of four warps ----------------
+    // Group g turns the 16-position blocks c = g, g+2, ... of every tile.  Inside a group, warp q
+    // reads tensor-memory lanes 32q.. (its quarter of the CTA's vocabulary entries) and stores them
+    // transposed; then thread (position i = tid & 15, vocabulary eighth e = tid >> 4) folds its 16 logits.
+    const int group = warp >> 2, q = warp & 3;
+    const int gtid = threadIdx.x & 127;              // thread index inside the group
+    const int pos_i = gtid & 15, eighth = gtid >> 4;
+    Stream st[kGroupChunks];
 #pragma unroll
-    for (int c = 0; c < kChunks; ++c) { st[c].mx = kMaskFloor; st[c].S = 0.f; st[c].u = 0.f; st[c].idx = kIdxNone; }
-    float* turn = reinterpret_cast<float*>(gbase + kOffTurn);
-    const int nchunks = (p.R + kChunk - 1) / kChunk;
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    for (int k = 0; k < kGroupChunks; ++k) { st[k].mx = kMaskFloor; st[k].S = 0.f; st[k].u = 0.f; st[k].idx = kIdxNone; }
+    float* turn = reinterpret_cast<float*>(gbase + kOffTurn + group * kTurnGroupBytes);
+    const int nchunks = (p.R + kChunk - 1) / kChunk;                 // blocks of this launch
+    const int my_chunks = nchunks > group ? (nchunks - group + 1) / 2 : 0;  // ... that this group turns
+    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
     for (int t = 0; t < my_tiles; ++t) {
-      if (threadIdx.x == 0) misc[1] = mbar_wait(tmem_full, t & 1, p.status, kErrTimeoutEpilogue) ? 1u : 0u;
-      epi_bar();
-      const bool go = misc[1] != 0;  // one thread waits, all take the same decision
+      if (gtid == 0) misc[1 + group] = mbar_wait(tmem_full, t & 1, p.status, kErrTimeoutEpilogue) ? 1u : 0u;
+      group_bar(group);
+      const bool go = misc[1 + group] != 0;  // one thread per group waits, the group takes the same decision
       if (!go) break;
       tc_fence_after();
-      const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + warp * 32;
-      const int limit = p.V - v0;  // entries of this quarter that exist
+      const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + eighth * 16;
+      const int limit = p.V - v0;  // entries of this eighth that exist
+      if (my_chunks == 0) {        // nothing to read for this group: hand the accumulators back at once
+        tc_fence_before();
+        mbar_arrive_remote(map_to_cta(tmem_empty, 0));
+      }
 #pragma unroll
-      for (int c = 0; c < kChunks; ++c) {
-        if (c < nchunks) {
-          uint32_t r[32];
-          tmem_ld32(tmem + lane_base + (uint32_t)(c * kChunk), r);
-          if (c == nchunks - 1) {  // last read of this tile: hand the accumulators back to the MMA issuer
+      for (int k = 0; k < kGroupChunks; ++k) {
+        if (k < my_chunks) {
+          const int c = 2 * k + group;
+          uint32_t r[16];
+          tmem_ld16(tmem + lane_base + (uint32_t)(c * kChunk), r);
+          if (k == my_chunks - 1) {  // last read of this tile by this thread: hand the accumulators back
             tc_fence_before();
             mbar_arrive_remote(map_to_cta(tmem_empty, 0));
           }
-          epi_bar();  // everyone is done reading the previous block
+          group_bar(group);  // the group is done reading the previous block
 #pragma unroll
-          for (int i = 0; i < 32; ++i) turn[i * kTurnRow + warp * 32 + lane] = __uint_as_float(r[i]);
-          epi_bar();
-          float x[32];
-          const float4* src = reinterpret_cast<const float4*>(turn + lane * kTurnRow + warp * 32);
+          for (int i = 0; i < 16; ++i) turn[i * kTurnRow + q * 32 + lane] = __uint_as_float(r[i]);
+          group_bar(group);
+          float x[16];
+          const float4* src = reinterpret_cast<const float4*>(turn + pos_i * kTurnRow + eighth * 16);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float4 q = src[j];
-            x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
+          for (int jj = 0; jj < 4; ++jj) {
+            const float4 v = src[jj];
+            x[4 * jj] = v.x; x[4 * jj + 1] = v.y; x[4 * jj + 2] = v.z; x[4 * jj + 3] = v.w;
           }
-          if (limit < 32) {  // ragged vocabulary: entries past V do not exist
+          if (limit < 16) {  // ragged vocabulary: entries past V do not exist
 #pragma unroll
-            for (int e = 0; e < 32; ++e)
+            for (int e = 0; e < 16; ++e)
               if (e >= limit) x[e] = kMaskFloor;
           }
-          fold32(st[c], x, v0);
+          fold16(st[k], x, v0);
         }
       }
     }
-    // Merge the four vocabulary quarters of every position and write the CTA's partial state.
+    // Merge the eight vocabulary eighths of every position and write the CTA's partial state.
     // The weight ring is free by now: every MMA that read it has completed (tmem_full of the last tile).
-    epi_bar();
+    epi_all_bar();
     Partial* buf = reinterpret_cast<Partial*>(gbase + kOffW);
 #pragma unroll
-    for (int c = 0; c < kChunks; ++c) {
-      Partial q;
-      q.mx = st[c].mx; q.S = st[c].S; q.u = st[c].u; q.idx = st[c].idx;
-      buf[(c * kChunk + lane) * 4 + warp] = q;
+    for (int k = 0; k < kGroupChunks; ++k) {
+      Partial pq;
+      pq.mx = st[k].mx; pq.S = st[k].S; pq.u = st[k].u; pq.idx = st[k].idx;
+      buf[((2 * k + group) * kChunk + pos_i) * 8 + eighth] = pq;
     }
-    epi_bar();
+    epi_all_bar();
     for (int pos = threadIdx.x; pos < p.R; pos += kEpiThreads) {
-      Partial a = buf[pos * 4];
-      merge_partial(a, buf[pos * 4 + 1]);
-      merge_partial(a, buf[pos * 4 + 2]);
-      merge_partial(a, buf[pos * 4 + 3]);
+      Partial a = buf[pos * 8];
+#pragma unroll
+      for (int e = 1; e < 8; ++e) merge_partial(a, buf[pos * 8 + e]);
       p.partials[(int64_t)(p.row0 + pos) * gridDim.x + blockIdx.x] = a;
     }
   }
