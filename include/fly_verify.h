@@ -176,6 +176,20 @@ fly_status_t fly_verify_reduce_shard(fly_verify_t* handle, int32_t rows, const v
 fly_status_t fly_verify_run_partials(fly_verify_t* handle, const fly_verify_args_t* args, const fly_partial_t* partials,
                                      int32_t world, int32_t total_vocab, void* cuda_stream);
 
+/* Prompt-lookup drafting: the step BEFORE verification.  Section 2.3 (multi-level acceleration) speeds
+ * the drafter up with prompt lookup decoding, "a simple n-gram retrieval method"; the paper gives no
+ * parameters, so the rule is the cited method's: the sequence's last n tokens are searched in its
+ * own earlier tokens, n from max_ngram down to min_ngram; at the first n with a match the EARLIEST
+ * match position p wins and the tokens that followed it, tokens[p+n .. p+n+K) cut at the sequence end,
+ * are proposed.
+ *   tokens   dev [B, stride] int32, sequence b holds lengths[b] <= stride tokens
+ *   draft    dev [B, K]: count[b] proposed tokens, then -1      count  dev [B] (0: no match)
+ *   match_pos / match_ngram   dev [B] or NULL: p (-1: none) and n (0: none)
+ * 1 <= min_ngram <= max_ngram <= 8.  No handle, no scratch; asynchronous on `cuda_stream`. */
+fly_status_t fly_pld_draft(int32_t device, int32_t B, const int32_t* tokens, int64_t stride, const int32_t* lengths,
+                           int32_t max_ngram, int32_t min_ngram, int32_t K, int32_t* draft, int32_t* count,
+                           int32_t* match_pos, int32_t* match_ngram, void* cuda_stream);
+
 /* The paper has no counterpart of this entry point; it exists for callers that
  * must not allocate device memory.
  *

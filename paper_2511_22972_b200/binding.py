@@ -22,6 +22,7 @@ FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
     "fly_verify_device_status", "fly_verify_selftest_wait", "fly_verify_reduce_shard", "fly_verify_run_partials",
+    "fly_pld_draft",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -85,6 +86,9 @@ def lib() -> C.CDLL:
     L.fly_verify_run_partials.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_void_p]
     L.fly_verify_run_partials.restype = C.c_int
+    L.fly_pld_draft.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.fly_pld_draft.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -222,6 +226,21 @@ def run_static(args: fly_verify_args_t, vocab: int, dtype: str = "bf16", device:
                                      C.byref(args), C.c_void_p(stream))
     if st != FLY_OK:
         raise FlyError(st, "fly_verify_run_static")
+
+
+def pld_draft(tokens, lengths, K: int, max_ngram: int = 3, min_ngram: int = 1, device: int = 0, stream: int = 0):
+    """fly_pld_draft on tokens [B, Lmax] int32 and lengths [B] int32 (device tensors).  Returns
+    (draft [B, K], count [B], match_pos [B], match_ngram [B]) as new device tensors."""
+    import torch
+    B = tokens.shape[0]
+    assert tokens.dtype == torch.int32 and lengths.dtype == torch.int32 and tokens.stride(1) == 1
+    draft = torch.empty(B, K, dtype=torch.int32, device=tokens.device)
+    count, pos, ng = (torch.empty(B, dtype=torch.int32, device=tokens.device) for _ in range(3))
+    st = lib().fly_pld_draft(int(device), int(B), _ptr(tokens), int(tokens.stride(0)), _ptr(lengths), int(max_ngram),
+                             int(min_ngram), int(K), _ptr(draft), _ptr(count), _ptr(pos), _ptr(ng), C.c_void_p(stream))
+    if st != FLY_OK:
+        raise FlyError(st, "fly_pld_draft")
+    return draft, count, pos, ng
 
 
 def static_args(*a, **kw) -> fly_verify_args_t:

@@ -13,6 +13,7 @@
 
 #include "fly_common.cuh"
 #include "lmhead_kernel.cuh"
+#include "pld_kernel.cuh"
 #include "reduce_kernel.cuh"
 #include "scan_kernel.cuh"
 
@@ -474,6 +475,21 @@ fly_status_t fly_verify_run_partials(fly_verify_t* h, const fly_verify_args_t* a
   if (e != cudaSuccess) return cuda_fail(h, e);
   h->last_launches = 2;
   return FLY_OK;
+}
+
+fly_status_t fly_pld_draft(int32_t device, int32_t B, const int32_t* tokens, int64_t stride, const int32_t* lengths,
+                           int32_t max_ngram, int32_t min_ngram, int32_t K, int32_t* draft, int32_t* count,
+                           int32_t* match_pos, int32_t* match_ngram, void* cuda_stream) {
+  if (device < 0 || B < 1 || !tokens || !lengths || !draft || !count || stride < 1) return FLY_ERR_INVALID_ARG;
+  if (min_ngram < 1 || max_ngram < min_ngram || max_ngram > fly::pld::kMaxNgram || K < 1) return FLY_ERR_INVALID_ARG;
+  DeviceGuard g(device);
+  if (!g.ok) return FLY_ERR_CUDA;
+  fly::pld::Params p;
+  p.tokens = tokens; p.stride = stride; p.lengths = lengths;
+  p.B = B; p.max_ngram = max_ngram; p.min_ngram = min_ngram; p.K = K;
+  p.draft = draft; p.count = count; p.match_pos = match_pos; p.match_ngram = match_ngram;
+  fly::pld::pld_draft_kernel<<<(unsigned)B, fly::pld::kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
+  return cudaGetLastError() == cudaSuccess ? FLY_OK : FLY_ERR_CUDA;
 }
 
 fly_status_t fly_verify_device_status(fly_verify_t* h, void* cuda_stream) {
