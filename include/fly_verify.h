@@ -16,6 +16,7 @@
  *     Position K+1 is the bonus position.
  *   - fly_verify_run is asynchronous on the given CUDA stream, allocates
  *     nothing and never synchronises the host with the device.
+ *   - A handle is not thread-safe: use one per host thread, or serialise the calls on it.
  *   - No function throws, aborts or traps.  Misuse that the host can see is
  *     reported by the return code before anything is launched; conditions that
  *     depend on device data (non-finite logits, draft ids out of range) are

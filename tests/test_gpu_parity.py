@@ -298,3 +298,68 @@ def test_caller_supplied_target_tokens():
                              state_in=None if state is None else np.asarray(state), target_tokens=tt.cpu().numpy())
         assert ref.row_flags[3, 2] == 4 and ref.row_flags[5, w.K] == 4
         assert_parity(out, ref, f"target tokens {boundary}")
+
+
+def _guarded(shape, dtype, fill):
+    """A tensor with 64 canary elements on either side of the part handed to the library."""
+    n = int(np.prod(shape))
+    raw = torch.full((n + 128,), fill, dtype=dtype, device=DEV)
+    return raw, raw[64:64 + n].view(*shape)
+
+
+def test_nothing_is_written_outside_the_output_buffers():
+    from paper_2511_22972_b200 import VerifyBuffers, verify, verify_fused
+    B, K = 5, 7
+    for fused in (False, True):
+        V = 32064 if not fused else 2048
+        out = VerifyBuffers(B, K, DEV)
+        raws = {}
+        for name, dtype, fill in [("accept_len", torch.int32, 12345), ("rollback", torch.int32, 12345),
+                                  ("out_tokens", torch.int32, 12345), ("target_argmax", torch.int32, 12345),
+                                  ("entropy", torch.float32, 777.0), ("row_flags", torch.int32, 12345),
+                                  ("state", torch.int32, 12345)]:
+            raw, view = _guarded(tuple(getattr(out, name).shape), dtype, fill)
+            raws[name] = (raw, fill)
+            setattr(out, name, view)
+        st = torch.cuda.current_stream().cuda_stream
+        if not fused:
+            w = small("bf16", B=B, K=K, V=V)
+            fv = FlyVerify(B, K, V, "bf16")
+            logits, draft = draw(w, step=31)
+            for splits in (0, 1, 5):
+                fv.set_splits(splits)
+                verify(fv, logits, draft, out, stream=st)
+        else:
+            w = S.shrink(S.FUSED, B=B, K=K, V=V, hidden=256, weight_std=0.1)
+            fv = FlyVerify(B, K, V, "bf16", hidden=256)
+            verify_fused(fv, S.make_hidden(w, 0, device=DEV), S.make_weight(w, device=DEV),
+                         torch.zeros(B, K, dtype=torch.int32, device=DEV), out, stream=st)
+        torch.cuda.synchronize()
+        for name, (raw, fill) in raws.items():
+            assert (raw[:64] == fill).all() and (raw[-64:] == fill).all(), f"{name}: canary overwritten (fused={fused})"
+        s = out.accept_len
+        assert ((s >= 1) & (s <= K + 1)).all()
+
+
+def test_a_captured_step_replays_correctly():
+    # fly_verify_run enqueues work only (no allocation, no synchronisation): it can be captured in a CUDA graph
+    from paper_2511_22972_b200 import VerifyBuffers, verify
+    w = small("bf16", B=8, K=8, V=128256)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    logits, draft = draw(w, step=41)
+    out = VerifyBuffers(w.B, w.K, DEV)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        verify(fv, logits, draft, out, stream=stream.cuda_stream)      # warm-up outside capture
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            verify(fv, logits, draft, out, stream=stream.cuda_stream)
+        logits2, draft2 = draw(w, step=42)
+        logits.copy_(logits2)                                          # new inputs in the captured buffers
+        draft.copy_(draft2)
+        out.accept_len.fill_(-1)
+        g.replay()
+        stream.synchronize()
+    torch.cuda.synchronize()
+    assert_parity(out, oracle_step(logits, draft, 1.0, 3), "graph replay")
