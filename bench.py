@@ -411,7 +411,7 @@ def main():
     if w.hidden:
         run_fused(args, w)
         return
-    args.steps = args.steps or max(2000, int(0.6 / (w.rows * w.V * w.elem_bytes / 6.0e12)))   # ~0.6 s of timed work
+    args.steps = args.steps or min(200000, max(2000, int(0.6 / (w.rows * w.V * w.elem_bytes / 6.0e12))))   # <= ~0.6 s of timed work
     args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
 
     import torch
