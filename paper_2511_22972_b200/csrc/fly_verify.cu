@@ -89,8 +89,9 @@ fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
 // fill the machine, and whole rows (or a few large pieces) are fastest.
 int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
   const int64_t sms = h->sm_count;
-  int64_t cap = row_bytes / 32768;  // keep >= 32 KB per block
+  int64_t cap = row_bytes / 32768;  // keep >= 32 KB per block ...
   if (cap < 1) cap = 1;
+  if (2 * rows * cap < sms && row_bytes / 16384 > cap) cap = row_bytes / 16384;  // ... 16 KB when the grid is far from filling the SMs
   if (cap > kMaxSplits) cap = kMaxSplits;
   if (cap > max_pieces) cap = max_pieces;
   if (h->overlap) {
