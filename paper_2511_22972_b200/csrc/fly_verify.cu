@@ -69,8 +69,8 @@ struct fly_verify {
   // staging for fly_verify_run_host (allocated on first use)
   void* st_logits = nullptr;
   size_t st_logits_bytes = 0;
-  int32_t* st_ints = nullptr;  // draft | state_in | state_out | accept | rollback | tokens | argmax | flags | target tokens
-  float* st_entropy = nullptr;
+  int32_t* st_ints = nullptr;  // device: draft | state_in | target tokens || state_out | accept | rollback | tokens | argmax | flags | entropy
+  int32_t* st_host = nullptr;  // page-locked host copy of the same block
 };
 
 namespace {
@@ -391,7 +391,7 @@ fly_status_t fly_verify_destroy(fly_verify_t* h) {
     cudaFree(h->st_hidden);
     cudaFree(h->st_logits);
     cudaFree(h->st_ints);
-    cudaFree(h->st_entropy);
+    cudaFreeHost(h->st_host);
   }
   delete h;
   return FLY_OK;
@@ -593,11 +593,12 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
   const int64_t stride = a->row_stride ? a->row_stride : V;
   cudaError_t e;
   if (!h->st_ints) {
-    // staging sized once for the largest run this handle allows
+    // staging sized once for the largest run this handle allows: the small inputs and all outputs are
+    // packed into one block each way, so that a step costs one small copy in and one out
     const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
-    const size_t ints = (size_t)(mb * (mk1 - 1) + 3 * mb + 3 * mb + mb + mb + 4 * mb * mk1);
-    if ((e = cudaMalloc(&h->st_ints, ints * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
-    if ((e = cudaMalloc(&h->st_entropy, (size_t)(mb * mk1) * sizeof(float))) != cudaSuccess) return cuda_fail(h, e);
+    const size_t words = (size_t)(mb * (mk1 - 1) + 3 * mb + mb * mk1) + (size_t)(3 * mb + mb + mb + 4 * mb * mk1);
+    if ((e = cudaMalloc(&h->st_ints, words * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMallocHost(&h->st_host, words * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
   }
   const size_t hidden_bytes = a->logits ? 0 : (size_t)rows * h->cfg.hidden * 2;
   if (hidden_bytes > h->st_hidden_bytes) {
@@ -615,57 +616,53 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     if ((e = cudaMalloc(&h->st_logits, logit_bytes)) != cudaSuccess) return cuda_fail(h, e);
     h->st_logits_bytes = logit_bytes;
   }
-  const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
-  int32_t* d_draft = h->st_ints;
-  int32_t* d_state_in = d_draft + mb * (mk1 - 1);
-  int32_t* d_state_out = d_state_in + 3 * mb;
-  int32_t* d_accept = d_state_out + 3 * mb;
-  int32_t* d_rollback = d_accept + mb;
-  int32_t* d_tokens = d_rollback + mb;
-  int32_t* d_argmax = d_tokens + mb * mk1;
-  int32_t* d_flags = d_argmax + mb * mk1;
-  int32_t* d_target = d_flags + mb * mk1;
+  // word offsets inside the staging block (same layout on the host and on the device)
+  const int64_t o_draft = 0, o_state_in = o_draft + B * a->K, o_target = o_state_in + 3 * B, in_words = o_target + rows;
+  const int64_t o_state_out = in_words, o_accept = o_state_out + 3 * B, o_rollback = o_accept + B,
+                o_tokens = o_rollback + B, o_argmax = o_tokens + rows, o_flags = o_argmax + rows,
+                o_entropy = o_flags + rows, all_words = o_entropy + rows;
+  int32_t* dv = h->st_ints;
+  int32_t* hv = h->st_host;
+  memcpy(hv + o_draft, a->draft, (size_t)(B * a->K) * 4);
+  if (a->state_in) memcpy(hv + o_state_in, a->state_in, (size_t)B * 12);
+  if (a->target_tokens) memcpy(hv + o_target, a->target_tokens, (size_t)rows * 4);
 
   if (a->logits && (e = cudaMemcpyAsync(h->st_logits, a->logits, logit_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
   if (!a->logits && (e = cudaMemcpyAsync(h->st_hidden, a->hidden, hidden_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
     return cuda_fail(h, e);
-  if ((e = cudaMemcpyAsync(d_draft, a->draft, (size_t)(B * a->K) * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-    return cuda_fail(h, e);
-  if (a->state_in &&
-      (e = cudaMemcpyAsync(d_state_in, a->state_in, (size_t)B * 12, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-    return cuda_fail(h, e);
-  if (a->target_tokens &&
-      (e = cudaMemcpyAsync(d_target, a->target_tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess)
-    return cuda_fail(h, e);
+  if ((e = cudaMemcpyAsync(dv, hv, (size_t)in_words * 4, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(h, e);
 
   fly_verify_args_t d = *a;
   d.logits = a->logits ? h->st_logits : nullptr;
   d.hidden = a->logits ? nullptr : h->st_hidden;  // the weight stays where it is: device memory
-  d.draft = d_draft;
-  d.state_in = a->state_in ? reinterpret_cast<const fly_state_t*>(d_state_in) : nullptr;
-  d.state_out = a->state_out ? reinterpret_cast<fly_state_t*>(d_state_out) : nullptr;
-  d.accept_len = d_accept;
-  d.rollback = a->rollback ? d_rollback : nullptr;
-  d.out_tokens = d_tokens;
-  d.target_argmax = a->target_argmax ? d_argmax : nullptr;
-  d.entropy = a->entropy ? h->st_entropy : nullptr;
-  d.row_flags = a->row_flags ? reinterpret_cast<uint32_t*>(d_flags) : nullptr;
-  d.target_tokens = a->target_tokens ? d_target : nullptr;
+  d.draft = dv + o_draft;
+  d.state_in = a->state_in ? reinterpret_cast<const fly_state_t*>(dv + o_state_in) : nullptr;
+  d.state_out = reinterpret_cast<fly_state_t*>(dv + o_state_out);
+  d.accept_len = dv + o_accept;
+  d.rollback = dv + o_rollback;
+  d.out_tokens = dv + o_tokens;
+  d.target_argmax = dv + o_argmax;
+  d.entropy = reinterpret_cast<float*>(dv + o_entropy);
+  d.row_flags = reinterpret_cast<uint32_t*>(dv + o_flags);
+  d.target_tokens = a->target_tokens ? dv + o_target : nullptr;
   s = fly_verify_run(h, &d, cuda_stream);
   if (s != FLY_OK) return s;
 
-  auto back = [&](void* dst, const void* src, size_t n) -> bool {
-    if (!dst) return true;
-    e = cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, st);
-    return e == cudaSuccess;
-  };
-  if (!back(a->accept_len, d_accept, (size_t)B * 4) || !back(a->rollback, d_rollback, (size_t)B * 4) ||
-      !back(a->out_tokens, d_tokens, (size_t)rows * 4) || !back(a->target_argmax, d_argmax, (size_t)rows * 4) ||
-      !back(a->entropy, h->st_entropy, (size_t)rows * 4) || !back(a->row_flags, d_flags, (size_t)rows * 4) ||
-      !back(a->state_out, d_state_out, (size_t)B * 12))
+  if ((e = cudaMemcpyAsync(hv + in_words, dv + in_words, (size_t)(all_words - in_words) * 4, cudaMemcpyDeviceToHost, st)) !=
+      cudaSuccess)
     return cuda_fail(h, e);
   if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return cuda_fail(h, e);
+  auto back = [&](void* dst, int64_t off, size_t bytes) {
+    if (dst) memcpy(dst, hv + off, bytes);
+  };
+  back(a->accept_len, o_accept, (size_t)B * 4);
+  back(a->rollback, o_rollback, (size_t)B * 4);
+  back(a->out_tokens, o_tokens, (size_t)rows * 4);
+  back(a->target_argmax, o_argmax, (size_t)rows * 4);
+  back(a->entropy, o_entropy, (size_t)rows * 4);
+  back(a->row_flags, o_flags, (size_t)rows * 4);
+  back(a->state_out, o_state_out, (size_t)B * 12);
   return FLY_OK;
 }
 
