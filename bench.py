@@ -280,6 +280,21 @@ def run_fused(args, w):
     d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
 
     flops = 2.0 * w.rows * w.hidden * w.V
+    # context only: the library GEMM (torch.matmul -> cuBLAS) on the SAME shape, writing bf16 logits, same
+    # number of back-to-back launches.  It does none of the verification; it shows what the shape allows.
+    lib_logits = torch.empty(w.rows, w.V, dtype=torch.bfloat16, device=device)
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            torch.matmul(hiddens[0], weight, out=lib_logits)
+        stream.synchronize()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l0.record(stream)
+        for i in range(args.steps):
+            torch.matmul(hiddens[i % nbuf], weight, out=lib_logits)
+        l1.record(stream)
+        stream.synchronize()
+    lib_ms = l0.elapsed_time(l1) / args.steps
+    del lib_logits
     burst, sustained, kind = measured_tensor_peak()
     achieved = flops / (ms_per_step * 1e-3) / 1e12
     line = {
@@ -297,6 +312,9 @@ def run_fused(args, w):
                      "note": "duration = whole step (GEMM kernel + acceptance-scan kernel, the latter ~3 us)",
                      "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
         "hbm_gbs": (w.hidden * w.V * 2 + w.rows * w.hidden * 2) / (ms_per_step * 1e-3) / 1e9,
+        "library_gemm_same_shape": {"ms_per_step": lib_ms, "tflops": flops / (lib_ms * 1e-3) / 1e12,
+                                    "note": "torch.matmul (cuBLAS) hidden x weight -> bf16 logits only, no verification; "
+                                            "context, timed after the main measurement"},
         "e2e": {"value": rows_all * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                 "api": "fly_verify_run_host (hidden states and drafts in pinned host buffers; weight resident)"},
