@@ -90,6 +90,20 @@ __device__ __forceinline__ Partial ld_partial_cg(const Partial* p) {
 __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, int lane, int* sm_y) {
   const int K = p.K, K1 = p.K + 1;
   uint64_t mism = 0, defer = 0;
+  // Issue the loads that do not depend on the partial states first (draft tokens, carried state):
+  // they are cold misses, and this is the tail of the step, where every dependent round trip counts.
+  int dr[2];
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int i = half * 32 + lane;
+    dr[half] = i < K ? p.draft[(int64_t)b * K + i] : 0;
+  }
+  int pend = 0, len = 0, corr = -1;
+  if (p.carry && p.state_in) {
+    pend = p.state_in[b * 3 + 0];
+    len = p.state_in[b * 3 + 1];
+    corr = p.state_in[b * 3 + 2];
+  }
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     const int i = half * 32 + lane;  // 0-based row of this sequence
@@ -118,7 +132,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
       }
       sm_y[i] = y;
       if (i < K) {
-        const int d = p.draft[(int64_t)b * K + i];
+        const int d = dr[half];
         if (d < 0 || d >= p.V) flag |= kFlagBadDraft;
         is_mism = (d != y) || flag;
         is_defer = (H >= p.theta_nats) && !flag;  // a flagged position is never kept
@@ -134,13 +148,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
   }
   __syncwarp();
 
-  int pend = 0, len = 0, corr = -1;
-  if (p.carry && p.state_in) {
-    pend = p.state_in[b * 3 + 0];
-    len = p.state_in[b * 3 + 1];
-    corr = p.state_in[b * 3 + 2];
-  }
-  __syncwarp();  // state_in may alias state_out: all lanes read before lane 0 writes
+  __syncwarp();  // state_in may alias state_out: all lanes have read it (above) before lane 0 writes
   const RoundOutcome o = decide_round(mism, defer, K, p.W, p.carry, pend, len);
 
 #pragma unroll
@@ -149,7 +157,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
     if (i < K1) {
       int tok = -1;
       if (o.revoke) tok = (i == 0) ? corr : -1;
-      else if (i < o.s - 1) tok = p.draft[(int64_t)b * K + i];
+      else if (i < o.s - 1) tok = dr[half];
       else if (i == o.s - 1) tok = sm_y[i];
       p.out_tokens[(int64_t)b * K1 + i] = tok;
     }
