@@ -363,3 +363,39 @@ def test_a_captured_step_replays_correctly():
         stream.synchronize()
     torch.cuda.synchronize()
     assert_parity(out, oracle_step(logits, draft, 1.0, 3), "graph replay")
+
+
+def test_seeded_fuzz_over_shapes_options_and_boundary_modes():
+    # 80 random small steps: shapes, dtypes, strides, thresholds, windows, split counts, scan modes, carried state
+    import random
+    rng = random.Random(2511)
+    for case in range(80):
+        dtype = rng.choice(["bf16", "f32"])
+        B, K = rng.randint(1, 9), rng.randint(1, 20)
+        V = rng.choice([3, 17, 64, 255, 1024, 4099, 9000, 33000])
+        w = small(dtype, B=B, K=K, V=V, draft_mix=(0.7, 0.2, 0.1))
+        theta = rng.choice([0.05, 0.5, 1.0, 2.5])
+        W = rng.randint(0, K)
+        boundary = rng.choice(["reject", "carry"])
+        logits, draft = draw(w, step=1000 + case, thetas=[theta], guard=V > 4)
+        pad = rng.choice([0, 0, 8, 24])
+        if pad:                                        # rows further apart than V elements
+            wide = torch.zeros(B, K + 1, V + pad, dtype=logits.dtype, device=DEV)
+            wide[:, :, :V] = logits
+            logits = wide[:, :, :V]
+        state = None
+        if boundary == "carry":
+            state = [[rng.randint(0, min(W, K)), rng.randint(1, K + 1), rng.randrange(V)] if rng.random() < 0.5
+                     else [0, 0, -1] for _ in range(B)]
+        fv = FlyVerify(B, K, V, dtype)
+        fv.set_splits(rng.choice([0, 0, 1, 2, 5]))
+        fv.set_scan_mode(rng.random() < 0.3)
+        what = f"fuzz {case}: {dtype} B={B} K={K} V={V} theta={theta} W={W} {boundary} pad={pad}"
+        if V <= 4:                                     # entropies may sit on the threshold: compare the row statistics only
+            out = gpu_step(fv, logits, draft, theta, W, boundary, state)
+            ref = oracle_step(logits, draft, theta, W, boundary, state)
+            assert np.array_equal(out.target_argmax.cpu().numpy(), ref.target_argmax), what
+            assert np.abs(out.entropy.cpu().numpy() - ref.entropy).max() <= 1e-4, what
+        else:
+            check(fv, logits, draft, theta, W, boundary=boundary, state=state, what=what)
+        fv.close()
