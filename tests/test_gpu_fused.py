@@ -183,3 +183,16 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
     assert fv.device_status(st) == Bd.FLY_OK                      # the record was cleared
     fv.close()
     run_and_check(4, 8, D=256, V=2048)
+
+
+def test_seeded_fuzz_over_fused_shapes():
+    import random
+    rng = random.Random(22972)
+    for case in range(24):
+        B, K = rng.randint(1, 24), rng.randint(1, 15)
+        D = 8 * rng.randint(8, 160)                      # 64 .. 1280, any multiple of 8 (ragged last k-block)
+        V = 8 * rng.randint(16, 3000)                    # 128 .. 24000 (ragged last vocabulary tile, few or many tiles)
+        theta, W = rng.choice([0.5, 1.0, 3.0]), rng.randint(0, K)
+        boundary = rng.choice(["reject", "carry"])
+        state = [[rng.randint(0, min(W, K)), 2, 5] for _ in range(B)] if boundary == "carry" else None
+        run_and_check(B, K, D, V, theta=theta, W=W, boundary=boundary, state=state, step=case)
