@@ -65,3 +65,19 @@ def test_null_arguments():
     assert L.fly_verify_run_host(None, None, None) == Bd.FLY_ERR_INVALID_ARG
     assert L.fly_verify_set_option(None, 0, 1) == Bd.FLY_ERR_INVALID_ARG
     assert L.fly_verify_last_launch_count(None) == 0
+
+
+def test_header_is_plain_c_and_cxx(tmp_path):
+    # the boundary has to be usable from C: the header compiles as strict C99 and as C++17
+    import shutil
+    import subprocess
+    src = tmp_path / "h.c"
+    src.write_text('#include "fly_verify.h"\nint main(void) { fly_verify_args_t a; (void)a; '
+                   'return sizeof(fly_partial_t) == 16 && sizeof(fly_state_t) == 12 ? 0 : 1; }\n')
+    inc = os.path.join(ROOT, "include")
+    if shutil.which("gcc"):
+        subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", inc, "-fsyntax-only", str(src)],
+                       check=True)
+    if shutil.which("g++"):
+        subprocess.run(["g++", "-std=c++17", "-Wall", "-Wextra", "-Werror", "-I", inc, "-fsyntax-only", "-x", "c++", str(src)],
+                       check=True)
