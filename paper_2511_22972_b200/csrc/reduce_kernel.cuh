@@ -165,25 +165,25 @@ __device__ __forceinline__ void fold_slice_f32(WarpAcc& a, float (&x)[UNROLL][4]
 }
 
 
-// Loads segments seg0 + j*32 + lane (j < UNROLL) of a row into registers; segments at or past
-// seg_end read as -inf.  A full slice takes the unpredicated path.
+// Loads UNROLL segments, 32 segments apart, starting at p (a lane's pointer into a full slice).
 template <int UNROLL>
-__device__ __forceinline__ void load_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ row, int seg0,
-                                           int seg_end, int lane, uint32_t fill) {
-  if (seg0 + UNROLL * 32 <= seg_end) {
+__device__ __forceinline__ void load_full_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ p) {
 #pragma unroll
-    for (int j = 0; j < UNROLL; ++j) {
-      const uint4 q = ld_stream(row + seg0 + j * 32 + lane);
-      w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-    }
-  } else {
+  for (int j = 0; j < UNROLL; ++j) {
+    const uint4 q = ld_stream(p + j * 32);  // constant offsets: one pointer per slice
+    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
+  }
+}
+// The same for a slice that runs past seg_end: segments at or past seg_end read as -inf.
+template <int UNROLL>
+__device__ __forceinline__ void load_ragged_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ row, int seg0,
+                                                  int seg_end, int lane, uint32_t fill) {
 #pragma unroll
-    for (int j = 0; j < UNROLL; ++j) {
-      const int s = seg0 + j * 32 + lane;
-      uint4 q = make_uint4(fill, fill, fill, fill);
-      if (s < seg_end) q = ld_stream(row + s);
-      w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-    }
+  for (int j = 0; j < UNROLL; ++j) {
+    const int s = seg0 + j * 32 + lane;
+    uint4 q = make_uint4(fill, fill, fill, fill);
+    if (s < seg_end) q = ld_stream(row + s);
+    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
   }
 }
 
@@ -312,9 +312,17 @@ reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nse
   acc_init(a);
   constexpr int kSlice = UNROLL * 32;
   constexpr uint32_t kFill = sizeof(T) == 2 ? kNegInf2 : 0xff800000u;
-  for (int s0 = seg_begin + warp * kSlice; s0 < seg_end; s0 += kReduceWarps * kSlice) {
+  constexpr int kStride = kReduceWarps * kSlice;
+  int s0 = seg_begin + warp * kSlice;
+  const uint4* ptr = rv + s0 + lane;
+  for (; s0 + kSlice <= seg_end; s0 += kStride, ptr += kStride) {  // full slices: no predicates
     uint32_t w[UNROLL][4];
-    load_slice<UNROLL>(w, rv, s0, seg_end, lane, kFill);
+    load_full_slice<UNROLL>(w, ptr);
+    fold_slice<T, UNROLL>(a, w, s0, lane);
+  }
+  if (s0 < seg_end) {  // at most one slice of a warp runs past the end of the piece
+    uint32_t w[UNROLL][4];
+    load_ragged_slice<UNROLL>(w, rv, s0, seg_end, lane, kFill);
     fold_slice<T, UNROLL>(a, w, s0, lane);
   }
   // ragged tail (fewer than kElems logits): last unit of the row, last warp
