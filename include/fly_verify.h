@@ -99,7 +99,8 @@ typedef struct {
    * pass that yields l_1..l_{K+1} (Section 2.1) - formed in fp32 on the tensor
    * cores and never stored.
    * hidden: dev [B*(K+1), hidden] bf16 row-major, 16-byte aligned.
-   * weight: dev [hidden, V] bf16 row-major (V contiguous), 16-byte aligned.
+   * weight: dev [hidden, V] bf16 row-major (V contiguous), 16-byte aligned
+   *         (or [V, hidden] with FLY_OPT_WEIGHT_LAYOUT = 1).
    * hidden and V must be multiples of 8 (fly_verify_create checks).  Positions
    * are processed 288 at a time; each block of 288 streams the weight once. */
   const void* hidden;
@@ -245,11 +246,15 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
  *                         kernel is still draining and waits for it to complete only before its
  *                         first write.  Only correct if the logits of this step were complete
  *                         before that previous kernel started (e.g. back-to-back steps over inputs
- *                         already in memory).  0 (default): plain stream order. */
+ *                         already in memory).  0 (default): plain stream order.
+ * FLY_OPT_WEIGHT_LAYOUT   fused path only.  0 (default): weight is [hidden, V] row-major (V contiguous).
+ *                         1: weight is [V, hidden] row-major (hidden contiguous), the layout in which
+ *                         linear layers are usually stored. */
 typedef enum {
   FLY_OPT_SPLITS = 0,
   FLY_OPT_SCAN_MODE = 1,
-  FLY_OPT_STREAM_OVERLAP = 2
+  FLY_OPT_STREAM_OVERLAP = 2,
+  FLY_OPT_WEIGHT_LAYOUT = 3
 } fly_option_t;
 fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
 

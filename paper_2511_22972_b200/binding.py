@@ -17,7 +17,7 @@ FLY_STATIC_MAX_BATCH, FLY_STATIC_MAX_PIECES = 1024, 16384
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
-FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP = range(3)
+FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP, FLY_OPT_WEIGHT_LAYOUT = range(4)
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
@@ -152,6 +152,11 @@ class FlyVerify:
 
     def set_scan_mode(self, separate_kernel: bool):
         self.set_option(FLY_OPT_SCAN_MODE, 1 if separate_kernel else 0)
+
+    def set_weight_layout(self, vocab_major: bool):
+        """Fused path: True if the weight is stored [V, hidden] (hidden contiguous), False for [hidden, V]."""
+        self.set_option(FLY_OPT_WEIGHT_LAYOUT, 1 if vocab_major else 0)
+        self.weight_vd = bool(vocab_major)
 
     def set_stream_overlap(self, on: bool):
         self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)
@@ -288,7 +293,8 @@ def verify_fused(fv: FlyVerify, hidden, weight, draft, out: VerifyBuffers, theta
     The logits hidden @ weight are formed and reduced inside the kernel and never stored."""
     B, K = draft.shape
     rows, D = hidden.shape
-    assert rows == B * (K + 1) and tuple(weight.shape) == (D, fv.vocab)
+    assert rows == B * (K + 1)
+    assert tuple(weight.shape) == ((fv.vocab, D) if getattr(fv, "weight_vd", False) else (D, fv.vocab))
     assert hidden.is_contiguous() and weight.is_contiguous()
     carry = boundary == "carry"
     a = fv.make_args(B, K, draft, out.accept_len, out.out_tokens, hidden=hidden, weight=weight, theta=theta,

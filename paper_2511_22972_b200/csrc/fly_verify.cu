@@ -59,6 +59,7 @@ struct fly_verify {
   fly::Partial* lm_folded = nullptr;    // [max_rows]: partial states folded over CTAs (fused path) or ranks
   int* lm_status = nullptr;             // device word: first bounded wait that ran out (sticky until read)
   int lm_pairs = 0;                     // CTA pairs that can be resident at once
+  int weight_vd = 0;                    // 0: weight [hidden, V]; 1: weight [V, hidden]
   PFN_cuTensorMapEncodeTiled encode_tiled = nullptr;
   CUtensorMap map_w, map_h;             // cached for (map_w_ptr, map_h_ptr, map_h_rows)
   const void* map_w_ptr = nullptr;
@@ -218,7 +219,9 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
   if ((reinterpret_cast<uintptr_t>(a->hidden) & 15u) || (reinterpret_cast<uintptr_t>(a->weight) & 15u))
     return FLY_ERR_UNSUPPORTED;  // TMA needs 16-byte aligned bases
   if (h->map_w_ptr != a->weight) {
-    if (!encode_map(h, &h->map_w, a->weight, (uint64_t)V, (uint64_t)D, (uint64_t)V * 2, 64)) return FLY_ERR_CUDA;
+    const bool ok = h->weight_vd ? encode_map(h, &h->map_w, a->weight, (uint64_t)D, (uint64_t)V, (uint64_t)D * 2, L::kBlockV)
+                                 : encode_map(h, &h->map_w, a->weight, (uint64_t)V, (uint64_t)D, (uint64_t)V * 2, 64);
+    if (!ok) return FLY_ERR_CUDA;
     h->map_w_ptr = a->weight;
   }
   if (h->map_h_ptr != a->hidden || h->map_h_rows != rows) {
@@ -238,6 +241,7 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     p.num_tiles = num_tiles;
     p.num_kb = (D + L::kBlockK - 1) / L::kBlockK;
     p.row0 = (int)row0;
+    p.w_kmajor = h->weight_vd;
     p.partials = h->lm_partials;
     p.status = h->lm_status;
     L::lmhead_verify_kernel<<<grid, L::kThreads, L::kSmemBytes, st>>>(h->map_w, h->map_h, p);
@@ -411,6 +415,11 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
     case FLY_OPT_STREAM_OVERLAP:
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->overlap = v;
+      return FLY_OK;
+    case FLY_OPT_WEIGHT_LAYOUT:
+      if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
+      h->weight_vd = v;
+      h->map_w_ptr = nullptr;  // the cached tensor map describes the other layout
       return FLY_OK;
   }
   return FLY_ERR_INVALID_ARG;

@@ -96,6 +96,7 @@ struct Params {
   int num_tiles;  // ceil(V / 256): tiles of the CTA pairs
   int num_kb;     // ceil(D / 64)
   int row0;       // first row of this launch in hidden / partials
+  int w_kmajor;   // 0: weight is [D, V] (vocabulary contiguous, MN-major A); 1: weight is [V, D] (K-major A)
   Partial* partials;  // [rows, gridDim.x]: one partial state per position and CTA
   int* status;        // 0, or the code of the first wait that ran out
 };
@@ -179,8 +180,8 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);  // groups of 8 rows 1024 bytes apart
 // Instruction descriptor: fp32 accumulator, bf16 A and B, A MN-major (vocabulary
 // contiguous), B K-major, M = 256 (the pair), N = n.
-__host__ __device__ constexpr uint32_t instr_desc(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool a_kmajor) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_kmajor ? 0u : 1u) << 15) | (0u << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(kPairV >> 4) << 24);
 }
 
@@ -281,8 +282,12 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
           if (rank == 0) mbar_expect_tx(full(s), 2 * kBytesW);  // both CTAs' bytes
           const uint32_t bar = map_to_cta(full(s), 0);
           const uint32_t dst = base + kOffW + s * kBytesW;
-          tma_load_2d(dst, &map_w, v0, kb * kBlockK, bar);
-          tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, bar);
+          if (p.w_kmajor) {  // [V, D]: one box of 128 entries x 64 dims, each entry's 64 dims contiguous
+            tma_load_2d(dst, &map_w, kb * kBlockK, v0, bar);
+          } else {           // [D, V]: two boxes of 64 entries x 64 dims, each dim's 64 entries contiguous
+            tma_load_2d(dst, &map_w, v0, kb * kBlockK, bar);
+            tma_load_2d(dst + kBytesWBox, &map_w, v0 + 64, kb * kBlockK, bar);
+          }
         }
       }
     }
@@ -313,14 +318,16 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     // busy with two 144-column MMAs per 16 hidden dims, so each accumulator has an issuer of its own.
     const int half = warp - kWarpMma;
     if (lane == 0 && rank == 0 && (half == 0 || p.n1 > 0)) {
-      const uint32_t idesc = instr_desc(half == 0 ? p.n0 : p.n1);
+      const uint32_t idesc = instr_desc(half == 0 ? p.n0 : p.n1, p.w_kmajor != 0);
       const uint32_t d_tmem = tmem + (uint32_t)(half * kHalfN);
       // Everything that changes from one MMA to the next is a 32-bit add: this thread has to issue one
       // MMA every ~70 cycles, so the loop is kept to a few instructions per MMA.
       // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden dims
       // 1024 bytes apart (stride offset); 16 hidden dims further = 16 rows of 128 bytes.
       // B, K-major: groups of 8 positions 1024 bytes apart; 16 hidden dims further = 32 bytes.
-      const uint32_t a_lo0 = desc_lo(base + kOffW, kBytesWBox);
+      // With the weight stored [V, D] A is K-major like B: 128 rows of 128 bytes, 16 dims further = 32 bytes.
+      const uint32_t a_lo0 = p.w_kmajor ? desc_lo(base + kOffW, 16) : desc_lo(base + kOffW, kBytesWBox);
+      const uint32_t a_step = p.w_kmajor ? (uint32_t)((kMmaK * 2) >> 4) : (uint32_t)((kMmaK * 128) >> 4);
       const uint32_t b_lo0 = desc_lo(base + kOffH + half * kBytesHHalf, 16);
       const uint32_t peer_delta = map_to_cta(bar0, 1) - bar0;  // same offset in the partner's shared memory
       int st = 0;
@@ -338,7 +345,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
 #pragma unroll
           for (int ks = 0; ks < kBlockK / kMmaK; ++ks) {
             const uint32_t acc = ks == 0 ? (uint32_t)(kb != 0) : 1u;
-            mma_bf16(d_tmem, a_lo + ks * ((kMmaK * 128) >> 4), b_lo + ks * ((kMmaK * 2) >> 4), kDescHi, idesc, acc);
+            mma_bf16(d_tmem, a_lo + ks * a_step, b_lo + ks * ((kMmaK * 2) >> 4), kDescHi, idesc, acc);
           }
           // the stage may be refilled, in both CTAs, once these MMAs have read it
           const uint32_t eb = empty(st);

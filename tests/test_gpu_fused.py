@@ -196,3 +196,22 @@ def test_seeded_fuzz_over_fused_shapes():
         boundary = rng.choice(["reject", "carry"])
         state = [[rng.randint(0, min(W, K)), 2, 5] for _ in range(B)] if boundary == "carry" else None
         run_and_check(B, K, D, V, theta=theta, W=W, boundary=boundary, state=state, step=case)
+
+
+@pytest.mark.parametrize("D,V", [(64, 128), (512, 4096), (200, 1000), (1024, 19000)])
+def test_weight_stored_vocabulary_major(D, V):
+    # the same step with the weight stored [V, hidden] (the usual layout of a linear layer's parameter)
+    B, K = 4, 8
+    w, hidden, weight, draft, logits = fused_case(B, K, D, V, step=7)
+    fv = FlyVerify(B, K, V, "bf16", hidden=D)
+    fv.set_weight_layout(True)
+    out = VerifyBuffers(B, K, DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    verify_fused(fv, hidden, weight.t().contiguous(), draft, out, stream=st)
+    assert fv.device_status(st) == Bd.FLY_OK
+    ref = O.verify_batch(logits.reshape(B, K + 1, V), draft.cpu().numpy(), 1.0, 3)
+    assert_parity(out, ref, f"[V, D] weight D={D} V={V}")
+    fv.set_weight_layout(False)                                   # and back, on the same handle
+    verify_fused(fv, hidden, weight, draft, out, stream=st)
+    torch.cuda.synchronize()
+    assert_parity(out, ref, f"[D, V] weight D={D} V={V}")

@@ -214,7 +214,7 @@ def test_api_misuse_returns_error_codes():
     fv.set_scan_mode(True)
     run()
     assert fv.last_launch_count == 2                         # reduction + stand-alone scan
-    for opt, val in [(0, 33), (0, -1), (1, 2), (2, 2), (2, -1), (9, 0)]:
+    for opt, val in [(0, 33), (0, -1), (1, 2), (2, 2), (2, -1), (3, 2), (9, 0)]:
         with pytest.raises(FlyError):
             fv.set_option(opt, val)
 
