@@ -546,23 +546,7 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   h->last_launches = 0;
   if (!a->logits) return run_fused(h, a, st);
 
-  fly::ScanParams p;
-  p.B = a->B; p.K = a->K; p.V = V; p.splits = h->last_splits;
-  p.partials = h->partials;
-  p.tickets = nullptr;
-  p.draft = a->draft;
-  p.theta_nats = theta_to_nats(h, a);
-  p.W = a->W > 64 ? 64 : a->W;
-  p.carry = a->boundary == FLY_BOUNDARY_CARRY;
-  p.state_in = reinterpret_cast<const int32_t*>(a->state_in);
-  p.state_out = reinterpret_cast<int32_t*>(a->state_out);
-  p.accept_len = a->accept_len;
-  p.rollback = a->rollback;
-  p.out_tokens = a->out_tokens;
-  p.target_argmax = a->target_argmax;
-  p.entropy = a->entropy;
-  p.row_flags = a->row_flags;
-  p.target_tokens = a->target_tokens;
+  fly::ScanParams p = scan_params(h, a, h->partials, h->last_splits);
 
   const bool fused_tail = h->scan_mode == 0;
   cudaError_t e;
@@ -748,23 +732,8 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
   const int64_t room = FLY_STATIC_MAX_PIECES / rows;  // >= 1
   if (splits > room) splits = (int)room;
 
-  fly::ScanParams p;
-  p.B = a->B; p.K = a->K; p.V = vocab; p.splits = splits;
-  p.partials = partials;
+  fly::ScanParams p = scan_params(&h, a, partials, splits);
   p.tickets = tickets;
-  p.draft = a->draft;
-  p.theta_nats = theta_to_nats(&h, a);
-  p.W = a->W > 64 ? 64 : a->W;
-  p.carry = a->boundary == FLY_BOUNDARY_CARRY;
-  p.state_in = reinterpret_cast<const int32_t*>(a->state_in);
-  p.state_out = reinterpret_cast<int32_t*>(a->state_out);
-  p.accept_len = a->accept_len;
-  p.rollback = a->rollback;
-  p.out_tokens = a->out_tokens;
-  p.target_argmax = a->target_argmax;
-  p.entropy = a->entropy;
-  p.row_flags = a->row_flags;
-  p.target_tokens = a->target_tokens;
 
   // The arrival counters must start at zero, whatever an earlier call left behind.
   cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4, st);
