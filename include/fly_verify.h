@@ -271,6 +271,12 @@ fly_status_t fly_verify_device_status(fly_verify_t* handle, void* cuda_stream);
  * next fly_verify_device_status reports FLY_ERR_TIMEOUT.  Nothing faults or hangs. */
 fly_status_t fly_verify_selftest_wait(fly_verify_t* handle, void* cuda_stream);
 
+/* Introspection, host only (no CUDA call): the number of pieces into which the logits path cuts every
+ * row of row_bytes bytes when `rows` rows are reduced on a device with sm_count SMs, with or without
+ * FLY_OPT_STREAM_OVERLAP.  1..32; 0 for invalid arguments.  (Rows shorter than 32 segments of 16 bytes
+ * and unaligned rows may get fewer pieces than this at run time.) */
+int32_t fly_verify_plan_splits(int32_t sm_count, int64_t rows, int64_t row_bytes, int32_t stream_overlap);
+
 /* Number of kernels the last fly_verify_run enqueued (for accounting). */
 int32_t fly_verify_last_launch_count(const fly_verify_t* handle);
 

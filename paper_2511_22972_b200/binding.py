@@ -22,7 +22,7 @@ FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP, FLY_OPT_WEIGHT_LAYOUT
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
     "fly_verify_device_status", "fly_verify_selftest_wait", "fly_verify_reduce_shard", "fly_verify_run_partials",
-    "fly_pld_draft",
+    "fly_pld_draft", "fly_verify_plan_splits",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
     L.fly_pld_draft.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.fly_pld_draft.restype = C.c_int
+    L.fly_verify_plan_splits.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int32]
+    L.fly_verify_plan_splits.restype = C.c_int32
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]

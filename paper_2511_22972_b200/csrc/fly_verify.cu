@@ -530,6 +530,14 @@ fly_status_t fly_verify_selftest_wait(fly_verify_t* h, void* cuda_stream) {
   return e == cudaSuccess ? FLY_OK : cuda_fail(h, e);
 }
 
+int32_t fly_verify_plan_splits(int32_t sm_count, int64_t rows, int64_t row_bytes, int32_t stream_overlap) {
+  if (sm_count < 1 || rows < 1 || row_bytes < 1) return 0;
+  fly_verify h;
+  h.sm_count = sm_count;
+  h.overlap = stream_overlap ? 1 : 0;
+  return auto_splits(&h, rows, row_bytes, kMaxSplits);
+}
+
 int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
 int32_t fly_verify_last_cuda_error(const fly_verify_t* h) { return h ? h->last_cuda_error : 0; }
 

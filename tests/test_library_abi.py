@@ -81,3 +81,22 @@ def test_header_is_plain_c_and_cxx(tmp_path):
     if shutil.which("g++"):
         subprocess.run(["g++", "-std=c++17", "-Wall", "-Wextra", "-Werror", "-I", inc, "-fsyntax-only", "-x", "c++", str(src)],
                        check=True)
+
+
+def test_split_planning_rule():
+    # host logic of the logits path: how many pieces a row is cut into (no GPU needed)
+    plan = Bd.lib().fly_verify_plan_splits
+    row = 128256 * 2                                   # one bf16 row of the Llama-3 vocabulary
+    assert plan(148, 144, row, 1) == 1                 # overlapped steps: whole rows
+    assert plan(148, 144, row, 0) == 4                 # a lone grid wants >= 3.5 blocks per SM, evenly
+    assert plan(148, 1088, row, 0) in (1, 2) and plan(148, 2304, 152064 * 2, 0) == 1
+    assert plan(148, 16, row, 0) == 7                  # few rows: as many 32 KB pieces as the row has
+    assert plan(148, 9, 32000 * 4, 0) == 7             # tiny step: down to 16 KB pieces
+    assert plan(148, 16, row, 1) == 3                  # overlapped, few rows: a quarter of the SMs is enough
+    assert plan(0, 1, 1, 0) == 0 and plan(148, 0, row, 0) == 0
+    for rows in (1, 3, 17, 144, 500, 5000):
+        for rb in (64, 4096, 40000, row, 10 * row):
+            for ov in (0, 1):
+                s = plan(148, rows, rb, ov)
+                assert 1 <= s <= 32
+                assert s == 1 or rb // s >= 16384      # pieces never shrink below 16 KB
