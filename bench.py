@@ -429,7 +429,9 @@ def main():
     if w.hidden:
         run_fused(args, w)
         return
-    args.steps = args.steps or min(200000, max(2000, int(0.6 / (w.rows * w.V * w.elem_bytes / 6.0e12))))   # <= ~0.6 s of timed work
+    # ~0.15 s of timed work by default: long enough for a dozen clock samples, short enough to be timed in the
+    # same regime as the copy that the HBM peak was measured with (a burst, best of 10)
+    args.steps = args.steps or min(200000, max(2000, int(0.15 / (w.rows * w.V * w.elem_bytes / 6.0e12))))
     args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
 
     import torch
