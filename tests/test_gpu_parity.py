@@ -399,3 +399,25 @@ def test_seeded_fuzz_over_shapes_options_and_boundary_modes():
         else:
             check(fv, logits, draft, theta, W, boundary=boundary, state=state, what=what)
         fv.close()
+
+
+def test_many_sequences_and_a_very_long_vocabulary():
+    # sizes at the far ends: 4096 sequences (16384 rows, one arrival counter each), and a 1M-entry vocabulary
+    w = small("bf16", B=4096, K=3, V=1000)
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    logits, draft = draw(w, step=51)
+    check(fv, logits, draft, 1.0, 2, what="B=4096")
+    check(fv, logits, draft, 1.0, 2, boundary="carry", state=[[b % 3, 2, 7] for b in range(w.B)], what="B=4096 carry")
+    fv.close()
+    V = (1 << 20) + 8
+    w = small("bf16", B=2, K=1, V=V)
+    fv = FlyVerify(w.B, w.K, V, "bf16")
+    logits, draft = draw(w, step=52)
+    for splits in (0, 1, 32):
+        fv.set_splits(splits)
+        check(fv, logits, draft, 1.0, 1, what=f"V=2^20+8 splits={splits}")
+    rows = logits.view(-1, V)
+    rows[1, :] = rows[1, 0]                      # a constant row: entropy = ln V exactly, argmax = 0 (first of all ties)
+    out = gpu_step(fv, logits, draft, 1.0, 1)
+    assert out.target_argmax.view(-1)[1].item() == 0
+    assert abs(out.entropy.view(-1)[1].item() - math.log(V)) < 1e-4
