@@ -16,7 +16,8 @@ Parity pins (tests/test_oracle_*.py): closed-form entropies (uniform, one-hot,
 single spike), shift invariance, scipy's softmax/entropy, brute-force
 enumeration of every (Delta, gate, W) pattern against the declarative form of
 the rule, the theta -> +inf and W = 0 limits stated in the paper's ablation
-text, and the chunking invariant for the cross-round carry extension.
+text, the chunking invariant for the cross-round carry extension, and
+hand-built rounds for invalid input (non-finite rows, token ids out of range).
 "Parity unpinned": nothing here says anything about real-model behaviour
 (tau, accuracy recovery); that needs weights and datasets.
 """

@@ -195,3 +195,91 @@ def test_caller_supplied_target_tokens_replace_the_argmax_in_eq2_and_in_the_outp
     assert got.out_tokens[1, 0] == tt[1, 0] and got.out_tokens[0, K] == y[0, K]
     assert got.row_flags[2, K] == O.FLAG_BAD_TARGET and got.out_tokens[2, K] == 0
     assert np.array_equal(got.target_argmax, y)            # the argmax is still reported as such
+
+
+# ---------------------------------------------------------------------------
+# Invalid input.  The paper does not treat it; the reading (a flagged position is a mismatch that the
+# gate never defers, so an invalid or placeholder token id can never be kept or emitted as a draft)
+# protects Eq. 2 and Eq. 6.  Every expected value below is written out by hand.  All rows are flat
+# unless stated (four equal logits: H = ln 4 = 1.386 nats, Defer at every threshold used; the argmax
+# of a flat row is token 0, the lowest index).
+# ---------------------------------------------------------------------------
+
+def _flat_rows(B, K1, V=4):
+    return np.zeros((B, K1, V))
+
+
+def test_nonfinite_row_cuts_the_round_even_when_its_placeholder_token_equals_the_draft():
+    # K = 3, theta = 0, W = 0: every valid mismatch would be deferred and accepted (no window to check).
+    # Position 2 holds a NaN: its row has no defined argmax, the reported token is the placeholder 0.
+    # The draft at position 2 is 0 as well - if the placeholder were compared like a real token the
+    # position would "match" and all four tokens would be appended.  It must cut at 2 instead.
+    x = _flat_rows(1, 4)
+    x[0, 1, 2] = np.nan
+    draft = np.array([[0, 0, 0]])
+    r = O.verify_batch(x, draft, theta=0.0, W=0)
+    assert r.row_flags.tolist() == [[0, O.FLAG_NONFINITE, 0, 0]]
+    assert r.accept_len.tolist() == [2]
+    assert r.out_tokens.tolist() == [[0, 0, -1, -1]]          # draft 1, then the placeholder at the cut
+    assert r.target_argmax[0, 1] == 0 and r.entropy[0, 1] == 0.0
+    # the same with +inf in the row, and with a row that has no finite entry at all
+    for bad_row in ([0.0, np.inf, 0.0, 0.0], [-np.inf] * 4):
+        x2 = _flat_rows(1, 4)
+        x2[0, 1] = bad_row
+        r2 = O.verify_batch(x2, draft, theta=0.0, W=0)
+        assert r2.row_flags.tolist() == [[0, O.FLAG_NONFINITE, 0, 0]]
+        assert r2.accept_len.tolist() == [2] and r2.out_tokens.tolist() == [[0, 0, -1, -1]]
+    # a partly masked row is NOT invalid: two entries left, H = ln 2, argmax = first finite maximum
+    x3 = _flat_rows(1, 4)
+    x3[0, 1] = [-np.inf, 0.0, -np.inf, 0.0]
+    r3 = O.verify_batch(x3, np.array([[0, 1, 0]]), theta=0.0, W=0)
+    assert r3.row_flags.tolist() == [[0, 0, 0, 0]] and r3.accept_len.tolist() == [4]
+    assert r3.target_argmax[0, 1] == 1 and abs(r3.entropy[0, 1] - math.log(2)) < 1e-12
+
+
+def test_out_of_range_draft_on_a_defer_row_with_a_clean_window_is_cut_not_kept():
+    # K = 4, W = 2, theta = 0.5 nats.  Position 2 proposes token 7 (V = 4): a mismatch on a flat (Defer) row
+    # whose window 3..4 is clean and fits (2 + 2 <= 4).  For a valid id Eq. 9 says Accept and the DRAFT token
+    # would be appended - here that would put id 7 into the text.  The reading cuts at 2 and emits y_2 = 0.
+    x = _flat_rows(2, 5)
+    draft = np.array([[0, 7, 0, 0],       # invalid id
+                      [0, 3, 0, 0]])      # control: a valid mismatch in the same place IS kept (accept all)
+    r = O.verify_batch(x, draft, theta=0.5, W=2)
+    assert r.row_flags.tolist() == [[0, O.FLAG_BAD_DRAFT, 0, 0, 0], [0, 0, 0, 0, 0]]
+    assert r.accept_len.tolist() == [2, 5]
+    assert r.out_tokens.tolist() == [[0, 0, -1, -1, -1], [0, 3, 0, 0, 0]]
+    # a negative id is out of range too
+    r2 = O.verify_batch(x[:1], np.array([[0, 0, -1, 0]]), theta=0.5, W=0)
+    assert r2.row_flags.tolist() == [[0, 0, O.FLAG_BAD_DRAFT, 0, 0]]
+    assert r2.accept_len.tolist() == [3] and r2.out_tokens.tolist() == [[0, 0, 0, -1, -1]]
+
+
+def test_out_of_range_caller_token_is_never_accepted_even_when_the_placeholder_equals_the_draft():
+    # Caller-supplied target tokens (extension).  Position 2's token is 9 (V = 4): flagged, replaced by the
+    # placeholder 0 - which equals the draft there.  theta = 0, W = 0 would accept any valid mismatch.
+    x = _flat_rows(1, 4)
+    tt = np.array([[0, 9, 0, 0]])
+    r = O.verify_batch(x, np.array([[0, 0, 0]]), theta=0.0, W=0, target_tokens=tt)
+    assert r.row_flags.tolist() == [[0, O.FLAG_BAD_TARGET, 0, 0]]
+    assert r.accept_len.tolist() == [2] and r.out_tokens.tolist() == [[0, 0, -1, -1]]
+    # an invalid BONUS token (position K+1) takes no part in Eq. 2: the round is accepted, the placeholder is emitted
+    r2 = O.verify_batch(x, np.array([[0, 0, 0]]), theta=0.0, W=0, target_tokens=np.array([[0, 0, 0, -5]]))
+    assert r2.row_flags.tolist() == [[0, 0, 0, O.FLAG_BAD_TARGET]]
+    assert r2.accept_len.tolist() == [4] and r2.out_tokens.tolist() == [[0, 0, 0, 0]]
+    # a non-finite row ignores what the caller drew for it (flag 1 only)
+    x3 = _flat_rows(1, 4)
+    x3[0, 0, 0] = np.nan
+    r3 = O.verify_batch(x3, np.array([[2, 0, 0]]), theta=0.0, W=0, target_tokens=np.array([[2, 0, 0, 0]]))
+    assert r3.row_flags.tolist() == [[O.FLAG_NONFINITE, 0, 0, 0]]
+    assert r3.accept_len.tolist() == [1] and r3.out_tokens.tolist() == [[0, -1, -1, -1]]
+
+
+def test_flagged_position_inside_a_carried_window_revokes_it():
+    # Carry extension: one window slot is still open (pending = 1, rollback_len = 3, correction = 2).  Position 1
+    # of this round holds a NaN and the draft there equals the placeholder 0: it must count as the mismatch that
+    # revokes the carried deferral (s = 1, rollback 3, the correction token), not as a match.
+    x = _flat_rows(1, 4)
+    x[0, 0, 3] = np.nan
+    r = O.verify_batch(x, np.array([[0, 0, 0]]), theta=0.0, W=1, boundary="carry", state_in=np.array([[1, 3, 2]]))
+    assert r.accept_len.tolist() == [1] and r.rollback.tolist() == [3]
+    assert r.out_tokens.tolist() == [[2, -1, -1, -1]] and r.state_out.tolist() == [[0, 0, -1]]
