@@ -6,13 +6,25 @@ match/gate bits, deferred-window scan, token emission - over one batch of
 synthetic logits and draft tokens, through the C ABI.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+                  [--shard batch|vocab] [--launch graph|stream] [--no-extra] [--no-cpu-baseline]
 
-N > 1: launched by torch.distributed.run, one rank per GPU; every rank verifies
-its own B sequences (sequences are independent: weak scaling, no data-path
-collective) and the job time is the max over ranks.
+Headline numbers (`value`, `ms_per_step`, `roofline.frac`) are taken in PLAIN STREAM ORDER: every step's
+kernel waits for the previous kernel in the stream before its first read, which is what a decode loop
+needs (each round's logits come from the kernel before it).  The same steps with `inputs_ready` (a step
+may read while the step before it drains; only valid over inputs that are already complete) are reported
+next to them as `overlapped`.
 
---impl reference times the fp64 CPU oracle (the only "reference implementation"
-of this method that exists here) on the host cores, on a bounded sample.
+With one GPU and no --no-extra the line also carries `workloads`: every synthetic workload timed the
+same way (serial and overlapped; the fused LM-head workload against the tensor roofline).
+
+N > 1: launched by torch.distributed.run, one rank per GPU.  --shard batch (default): every rank verifies
+its own B sequences (sequences are independent: weak scaling, no data-path collective).  --shard vocab:
+every rank reduces its slice of the vocabulary, the 16-byte row states are all-gathered (NCCL) and every
+rank applies the acceptance rule (a tensor-parallel LM head; strong scaling).  The job time is the max
+over ranks.
+
+--impl reference times the fp64 CPU oracle (the only "reference implementation" of this method that
+exists here) on the host cores, on a bounded sample.
 """
 from __future__ import annotations
 
@@ -30,32 +42,41 @@ if ROOT not in sys.path:
 
 METRIC = "loose-verify positions/s and HBM GB/s (% of B200 peak) at V=128256 bf16"
 UNIT = "positions/s"
-FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+FALLBACK_HBM_GBS = 6650.0          # used only if MEASURED_PEAKS.json is absent
+FALLBACK_TENSOR = (1590.0, 1400.0)
 L2_BYTES = 126 * 1024 * 1024
+MIN_TIMED_S = 0.05                 # every timed region lasts at least this long
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the row-reduction kernel, from the ncu
-# captures summarised under profiles/ (bytes); None where no capture exists.
-NCU_TRAFFIC_BYTES = {
-    "long_draft_batch": 282.8e6,                        # measured: 279.14 MB read + 3.67 MB written
-    "llama3_vocab_batch": 282.8e6 * 144 / 1088,         # the same kernel; traffic scales with the rows read
-    "high_batch_serving": 282.8e6 * (2304 * 152064) / (1088 * 128256),
-    "fused_lm_head": (1.0675e9 + 4.4e6) * 128256 / 64000,   # measured at V = 64000; scales with V
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (bytes), keyed by kernel; None where the kernel has changed since its counters were taken.
+NCU_TRAFFIC = {
+    # reduce_rows_flat, long_draft_batch (1088 rows x 128256 bf16): see profiles/reduce_rows_flat_long_draft_batch.md
+    "reduce_rows_flat": None,
+    # lmhead_verify_kernel at V = 64000: see profiles/lmhead_verify_kernel_fused_lm_head.md
+    "lmhead_verify_kernel": None,
 }
 
 
-def measured_hbm_peak():
+def ncu_traffic(kernel, scale):
+    t = NCU_TRAFFIC.get(kernel)
+    return None if t is None else t["bytes"] * scale / t["units"]
+
+
+def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(p) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            d = json.load(f)
+        return {"hbm": float(d["hbm_gbs"]), "burst": float(d["bf16_tflops"]),
+                "sustained": float(d["bf16_tflops_sustained"]), "kind": "measured"}
     except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
+        return {"hbm": FALLBACK_HBM_GBS, "burst": FALLBACK_TENSOR[0], "sustained": FALLBACK_TENSOR[1], "kind": "fallback"}
 
 
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.index, self.period = index, period_s
         self.sm, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -109,38 +130,38 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.sm)}
 
 
-def build_inputs(w, device, nbuf):
-    """nbuf distinct (logits, draft) pairs resident on the device.  No entropy guard here: timing does
-    not need gate decisions to be precision-proof (the parity tests draw guarded inputs)."""
-    import torch
-    from paper_2511_22972_b200 import synthetic as S
-    bufs = []
-    for i in range(nbuf):
-        logits = S.make_logits(w, i, device=device)
-        draft = S.make_draft(w, i, S.rank5(logits.view(-1, w.V)))
-        bufs.append((logits, draft))
-    torch.cuda.synchronize()
-    return bufs
+# ------------------------------------------------------------------------------------------------------
+# timing
+# ------------------------------------------------------------------------------------------------------
 
-
-def time_steps(fv, arglist, stream, steps, warmup, ranks, launch):
-    """Device time of `steps` back-to-back steps: CUDA events on the launching stream, barrier and
-    synchronize on both sides, max over ranks.  Returns milliseconds for all steps."""
+def time_calls(call, n_args, stream, steps, warmup, ranks, launch):
+    """Device time of exactly `steps` back-to-back calls call(i % n_args): CUDA events on the launching
+    stream, barrier and synchronize on both sides, max over ranks.  launch == "graph": the calls are
+    captured once into CUDA graphs (one of up to 8 * n_args steps, replayed, plus one for the remainder),
+    so that the host's launch cost is out of the measurement.  Returns milliseconds for all steps."""
     import torch
     from paper_2511_22972_b200 import dist as D
-    n = len(arglist)
-    raw = stream.cuda_stream
     with torch.cuda.stream(stream):
         for i in range(max(warmup, 3)):
-            fv.run(arglist[i % n], raw)
-        graph, per_graph = None, 0
+            call(i % n_args)
+        stream.synchronize()
+        graphs = []
         if launch == "graph":
-            per_graph = min(steps, 8 * n)
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                for i in range(per_graph):
-                    fv.run(arglist[i % n], raw)
-            graph.replay()
+            per = min(steps, 8 * n_args)
+            reps, rem = divmod(steps, per)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for i in range(per):
+                    call(i % n_args)
+            graphs = [(g, reps)]
+            if rem:
+                g2 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g2, stream=stream):
+                    for i in range(rem):
+                        call(i % n_args)
+                graphs.append((g2, 1))
+            for g_, _ in graphs:
+                g_.replay()
         stream.synchronize()
         D.barrier(ranks)
         torch.cuda.synchronize()
@@ -148,62 +169,224 @@ def time_steps(fv, arglist, stream, steps, warmup, ranks, launch):
         e1 = torch.cuda.Event(enable_timing=True)
         torch.cuda.nvtx.range_push("fly_timed_region")      # lets a profiler list exactly the timed launches
         e0.record(stream)
-        if graph is not None:
-            done = 0
-            while done < steps:
-                graph.replay()
-                done += per_graph
-            steps_run = done
+        if graphs:
+            for g_, reps in graphs:
+                for _ in range(reps):
+                    g_.replay()
         else:
             for i in range(steps):
-                fv.run(arglist[i % n], raw)
-            steps_run = steps
+                call(i % n_args)
         e1.record(stream)
         torch.cuda.nvtx.range_pop()
         stream.synchronize()
         torch.cuda.synchronize()
         D.barrier(ranks)
-    ms = e0.elapsed_time(e1) * (steps / steps_run)
-    return D.max_over_ranks(ranks, ms)
+    return D.max_over_ranks(ranks, e0.elapsed_time(e1))
+
+
+def steps_for(step_s_estimate, asked):
+    """The step count of a timed region: what was asked for, else enough for MIN_TIMED_S."""
+    if asked:
+        return asked
+    return int(min(200000, max(50, MIN_TIMED_S * 1.5 / step_s_estimate)))
+
+
+def build_inputs(w, device, nbuf, near_miss=True):
+    """nbuf distinct (logits, draft) pairs resident on the device.  No entropy guard here: timing does
+    not need gate decisions to be precision-proof (the parity tests draw guarded inputs)."""
+    import torch
+    from paper_2511_22972_b200 import synthetic as S
+    bufs = []
+    for i in range(nbuf):
+        logits = S.make_logits(w, i, device=device)
+        rows = logits.view(-1, w.V)
+        top = S.rank5(rows) if (near_miss and w.draft_mix[1] > 0) else rows.float().argmax(dim=1, keepdim=True)
+        bufs.append((logits, S.make_draft(w, i, top)))
+    torch.cuda.synchronize()
+    return bufs
+
+
+def bench_logits(w, ranks, device, steps, warmup, launch, peaks, near_miss=True):
+    """One logits-path workload: serial (plain stream order) and overlapped (inputs_ready) step times."""
+    import torch
+    from paper_2511_22972_b200 import FlyVerify, VerifyBuffers
+    step_bytes = w.rows * w.V * w.elem_bytes
+    nbuf = max(2, -(-int(2.4 * L2_BYTES) // step_bytes))     # rotate over > 2x L2 of distinct inputs
+    bufs = build_inputs(w, device, nbuf, near_miss)
+    out = VerifyBuffers(w.B, w.K, device)
+    fv = FlyVerify(w.B, w.K, w.V, w.dtype, device=ranks.local_rank)
+    carry = w.boundary == "carry"
+
+    def mk(l, d, ready):
+        return fv.make_args(w.B, w.K, d, out.accept_len, out.out_tokens, logits=l, theta=w.theta, W=w.W,
+                            boundary=w.boundary, state_in=out.state if carry else None, state_out=out.state,
+                            rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
+                            row_flags=out.row_flags, inputs_ready=ready)
+
+    serial_args = [mk(l, d, False) for l, d in bufs]
+    ready_args = [mk(l, d, True) for l, d in bufs]
+    stream = torch.cuda.Stream(device=device)
+    raw = stream.cuda_stream
+    n = steps_for(max(step_bytes / (peaks["hbm"] * 1e9), 4e-6), steps)
+    res = {"steps": n, "nbuf": nbuf, "step_bytes": step_bytes}
+    with ClockSampler(ranks.local_rank) as clk:
+        res["serial_ms"] = time_calls(lambda i: fv.run(serial_args[i], raw), nbuf, stream, n, warmup, ranks, launch) / n
+        res["launches_per_step"] = fv.last_launch_count
+    res["clocks"] = clk.summary()
+    with ClockSampler(ranks.local_rank) as clk2:
+        res["overlapped_ms"] = time_calls(lambda i: fv.run(ready_args[i], raw), nbuf, stream, n, warmup, ranks, launch) / n
+    res["clocks_overlapped"] = clk2.summary()
+    res.update(fv=fv, bufs=bufs, stream=stream, carry=carry)
+    return res
+
+
+def logits_row(w, r, peaks, world):
+    """The `workloads` entry of a logits-path workload."""
+    gbs = lambda ms: r["step_bytes"] / (ms * 1e-3) / 1e9
+    return {
+        "rows_per_step": w.rows, "bytes_per_step": r["step_bytes"], "steps": r["steps"],
+        "us_per_step_serial": r["serial_ms"] * 1e3, "us_per_step_overlapped": r["overlapped_ms"] * 1e3,
+        "positions_per_s_serial": w.rows * world / (r["serial_ms"] * 1e-3),
+        "positions_per_s_overlapped": w.rows * world / (r["overlapped_ms"] * 1e-3),
+        "gbs_serial": gbs(r["serial_ms"]), "gbs_overlapped": gbs(r["overlapped_ms"]),
+        "frac_serial": gbs(r["serial_ms"]) / peaks["hbm"], "frac_overlapped": gbs(r["overlapped_ms"]) / peaks["hbm"],
+        "clocks": r["clocks"], "clocks_overlapped": r["clocks_overlapped"],
+    }
+
+
+def h2d_bandwidth(device, nbytes, stream):
+    """Pinned host -> device copy bandwidth for a buffer of nbytes (GB/s), best of 5: what bounds `e2e`."""
+    import torch
+    n = max(int(nbytes), 1 << 20)
+    src = torch.empty(n, dtype=torch.uint8).pin_memory()
+    dst = torch.empty(n, dtype=torch.uint8, device=device)
+    best = 0.0
+    with torch.cuda.stream(stream):
+        for _ in range(6):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            dst.copy_(src, non_blocking=True)
+            e1.record(stream)
+            stream.synchronize()
+            best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    return best
+
+
+def e2e_logits(w, r, ranks, device, steps_hint):
+    """The same metric end to end through fly_verify_run_host: logits and drafts start in pinned host
+    memory every step, results end in host memory, the call synchronises.  Wall clock, max over ranks."""
+    import torch
+    from paper_2511_22972_b200 import VerifyBuffers, dist as D
+    fv, bufs, stream, carry = r["fv"], r["bufs"], r["stream"], r["carry"]
+    step_bytes = r["step_bytes"]
+    h2d_gbs = h2d_bandwidth(device, step_bytes, stream)
+    est = step_bytes / (h2d_gbs * 1e9) + 30e-6
+    e2e_steps = int(max(10, min(400, 0.1 / est)))
+    host_l = [b[0].cpu().pin_memory() for b in bufs[:2]]
+    host_d = [b[1].cpu().pin_memory() for b in bufs[:2]]
+    hout = VerifyBuffers(w.B, w.K, device, pinned=True)
+    hargs = [fv.make_args(w.B, w.K, d, hout.accept_len, hout.out_tokens, logits=l, theta=w.theta, W=w.W,
+                          boundary=w.boundary, state_in=hout.state if carry else None, state_out=hout.state,
+                          rollback=hout.rollback, target_argmax=hout.target_argmax, entropy=hout.entropy,
+                          row_flags=hout.row_flags) for l, d in zip(host_l, host_d)]
+    raw = stream.cuda_stream
+    for i in range(3):
+        fv.run_host(hargs[i % 2], raw)
+    D.barrier(ranks)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        fv.run_host(hargs[i % 2], raw)          # synchronises the stream before returning
+    torch.cuda.synchronize()
+    e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
+    h2d = step_bytes + w.B * w.K * 4 + (w.B * 12 if carry else 0)
+    d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
+    value = w.rows * ranks.world * e2e_steps / e2e_s
+    bound = w.rows * ranks.world / (h2d / (h2d_gbs * 1e9))
+    return {"value": value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+            "us_per_step": e2e_s / e2e_steps * 1e6,
+            "h2d_gbs_measured": h2d_gbs, "bound": "pcie h2d copy of the step's logits",
+            "bound_value": bound, "frac_of_bound": value / bound,
+            "api": "fly_verify_run_host (pinned host buffers)"}
+
+
+# ------------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------------
+
+_BARRIER = None
+
+
+def _pool_init(barrier):
+    global _BARRIER
+    _BARRIER = barrier
+    import torch
+    torch.set_num_threads(1)
+
+
+def _oracle_worker(job):
+    """One worker process of the CPU baseline.  It draws its own share of the step (same recipe, its own
+    seed; untimed), waits until every worker is ready, then runs the oracle as it stands.  Returns the
+    system-wide monotonic clock at the start and at the end of the oracle call."""
+    import numpy as np
+    from oracle import fly_oracle as O
+    from paper_2511_22972_b200 import synthetic as S
+    ws, step = job
+    logits = S.make_logits(ws, step, device="cpu")
+    rows = logits.view(-1, ws.V)
+    top = S.rank5(rows) if ws.draft_mix[1] > 0 else rows.float().argmax(dim=1, keepdim=True)
+    d = S.make_draft(ws, step, top).numpy()
+    x = logits.double().numpy()
+    st = np.array([[0, 0, -1]] * ws.B) if ws.boundary == "carry" else None
+    _BARRIER.wait()
+    t0 = time.perf_counter()
+    O.verify_batch(x, d, ws.theta, ws.W, boundary=ws.boundary, state_in=st)
+    return t0, time.perf_counter()
+
+
+class OraclePool:
+    """The fp64 oracle on all host cores: sequences are independent, so every core verifies its own few
+    sequences of the workload's recipe with the (single-threaded, untouched) oracle, all at the same time.
+    One round's time is the wall clock from the first worker's start to the last worker's end."""
+
+    def __init__(self, w, rows_per_core):
+        import multiprocessing as mp
+        from paper_2511_22972_b200 import synthetic as S
+        cores = len(os.sched_getaffinity(0))
+        self.share = max(1, min(-(-w.B // cores), rows_per_core // (w.K + 1)))   # sequences per worker and round
+        self.workers = max(1, min(cores, w.B // self.share))
+        self.ws = S.shrink(w, B=self.share)
+        ctx = mp.get_context("fork")
+        self.pool = ctx.Pool(self.workers, initializer=_pool_init, initargs=(ctx.Barrier(self.workers),))
+        self.rows_per_round = self.workers * self.ws.rows
+        self.w = w
+
+    def round(self, step):
+        spans = self.pool.map(_oracle_worker, [(self.ws, step * self.workers + i) for i in range(self.workers)], chunksize=1)
+        return max(t1 for _, t1 in spans) - min(t0 for t0, _ in spans)
+
+    def sample(self, rounds):
+        return (f"{rounds} rounds of {self.workers} worker processes x {self.share} of {self.w.B} sequences x "
+                f"{self.ws.K + 1} rows x V={self.ws.V} ({self.w.dtype} widened to fp64)")
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
 
 
 def oracle_rate(w, seconds_budget=12.0):
-    """The fp64 oracle as it stands, on this host's cores, on whole steps of the workload drawn by the
-    same generator, until the budget is used (at least one step, or a row sample if one step is too long)."""
-    import numpy as np
-    import torch
-    from oracle import fly_oracle as O
-    from paper_2511_22972_b200 import synthetic as S
-    torch.set_num_threads(1)
-    rows_done, t_used, steps = 0, 0.0, 0
-    B = w.B
-    # bound one sample to ~150 rows so that a single call stays within seconds
-    if w.rows > 160:
-        B = max(1, 160 // (w.K + 1))
-    ws = S.shrink(w, B=B)
-    while t_used < seconds_budget:
-        logits = S.make_logits(ws, steps, device="cpu")
-        draft = S.make_draft(ws, steps, S.rank5(logits.view(-1, ws.V)))
-        x = logits.double().numpy()
-        d = draft.numpy()
-        t0 = time.perf_counter()
-        O.verify_batch(x, d, w.theta, w.W, boundary=w.boundary,
-                       state_in=np.array([[0, 0, -1]] * ws.B) if w.boundary == "carry" else None)
-        t_used += time.perf_counter() - t0
-        rows_done += ws.rows
-        steps += 1
-    return rows_done / t_used, f"{steps} steps of {ws.B} sequences x {ws.K + 1} rows x V={ws.V} ({w.dtype} widened to fp64)", 1
-
-
-def measured_tensor_peak():
-    """(burst, sustained) bf16 TFLOP/s of this machine's B200s, and where the numbers come from."""
-    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    """rows/s of the oracle on this host's cores, a description of the sample, and the cores used."""
+    op = OraclePool(w, rows_per_core=40)
     try:
-        with open(p) as f:
-            d = json.load(f)
-        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
-    except Exception:
-        return 1590.0, 1400.0, "fallback"
+        op.round(10 ** 6)                                   # untimed: pages in the workers
+        rows_done, t_used, rounds = 0, 0.0, 0
+        while t_used < seconds_budget:
+            t_used += op.round(rounds)
+            rows_done += op.rows_per_round
+            rounds += 1
+        return rows_done / t_used, op.sample(rounds), op.workers
+    finally:
+        op.close()
 
 
 def fused_oracle_sample(w, weight_cpu, seq, step):
@@ -229,16 +412,14 @@ def fused_oracle_sample(w, weight_cpu, seq, step):
     return t, ws.rows
 
 
-def run_fused(args, w):
-    """The fused LM-head workload: hidden [B*(K+1), D] x weight [D, V] with the verification in the epilogue."""
+# ------------------------------------------------------------------------------------------------------
+# fused LM-head workload
+# ------------------------------------------------------------------------------------------------------
+
+def bench_fused(w, ranks, device, steps, warmup, peaks, e2e=True, library=True):
+    """hidden [B*(K+1), D] x weight [D, V] with the verification in the epilogue; tensor roofline."""
     import torch
     from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, binding as Bd, dist as D, synthetic as S
-    args.steps = args.steps or 200
-    args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
-    ranks = D.init_from_env("nccl")
-    assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
-    torch.cuda.set_device(ranks.local_rank)
-    device = torch.device("cuda", ranks.local_rank)
     weight = S.make_weight(w, device=device)
     nbuf = 4
     hiddens = [S.make_hidden(w, i, device=device) for i in range(nbuf)]
@@ -252,85 +433,184 @@ def run_fused(args, w):
                                       target_argmax=o.target_argmax, entropy=o.entropy, row_flags=o.row_flags)
     arglist = [mk(h, d, out) for h, d in zip(hiddens, drafts)]
     stream = torch.cuda.Stream(device=device)
-    with ClockSampler(ranks.local_rank) as clk:
-        ms_total = time_steps(fv, arglist, stream, args.steps, args.warmup, ranks, "stream")
-        launches_per_step = fv.last_launch_count
-    if fv.device_status(stream.cuda_stream) != Bd.FLY_OK:
-        raise SystemExit("a bounded device-side wait ran out: the measurement is void")
-    ms_per_step = ms_total / args.steps
-    rows_all = w.rows * ranks.world
-    value = rows_all / (ms_per_step * 1e-3)
-
-    # end to end: hidden states and drafts come from pinned host memory every step, results go back
-    e2e_steps = max(10, min(100, args.steps // 2))
-    hout = VerifyBuffers(w.B, w.K, device, pinned=True)
-    hargs = [mk(h.cpu().pin_memory(), d.cpu().pin_memory(), hout) for h, d in zip(hiddens[:2], drafts[:2])]
-    keep = [a for a in hargs]
     raw = stream.cuda_stream
-    for i in range(3):
-        fv.run_host(hargs[i % 2], raw)
-    D.barrier(ranks)
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        fv.run_host(hargs[i % 2], raw)
-    torch.cuda.synchronize()
-    e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
-    h2d = w.rows * w.hidden * 2 + w.B * w.K * 4
-    d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
-
     flops = 2.0 * w.rows * w.hidden * w.V
-    # context only: the library GEMM (torch.matmul -> cuBLAS) on the SAME shape, writing bf16 logits, same
-    # number of back-to-back launches.  It does none of the verification; it shows what the shape allows.
-    lib_logits = torch.empty(w.rows, w.V, dtype=torch.bfloat16, device=device)
-    with torch.cuda.stream(stream):
-        for _ in range(3):
-            torch.matmul(hiddens[0], weight, out=lib_logits)
-        stream.synchronize()
-        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        l0.record(stream)
-        for i in range(args.steps):
-            torch.matmul(hiddens[i % nbuf], weight, out=lib_logits)
-        l1.record(stream)
-        stream.synchronize()
-    lib_ms = l0.elapsed_time(l1) / args.steps
-    del lib_logits
-    burst, sustained, kind = measured_tensor_peak()
-    achieved = flops / (ms_per_step * 1e-3) / 1e12
+    n = steps_for(flops / (peaks["burst"] * 1e12), steps)
+    with ClockSampler(ranks.local_rank) as clk:
+        ms = time_calls(lambda i: fv.run(arglist[i], raw), nbuf, stream, n, warmup, ranks, "stream") / n
+        launches_per_step = fv.last_launch_count
+    if fv.device_status(raw) != Bd.FLY_OK:
+        raise SystemExit("a bounded device-side wait ran out: the measurement is void")
+    achieved = flops / (ms * 1e-3) / 1e12
+    res = {"steps": n, "ms": ms, "flops": flops, "tflops": achieved, "launches_per_step": launches_per_step,
+           "clocks": clk.summary(), "frac_of_burst": achieved / peaks["burst"],
+           "frac_of_sustained": achieved / peaks["sustained"],
+           "hbm_gbs": (w.hidden * w.V * 2 + w.rows * w.hidden * 2) / (ms * 1e-3) / 1e9}
+    if e2e:
+        # end to end: hidden states and drafts come from pinned host memory every step, results go back
+        e2e_steps = max(10, min(100, n // 2))
+        hout = VerifyBuffers(w.B, w.K, device, pinned=True)
+        hargs = [mk(h.cpu().pin_memory(), d.cpu().pin_memory(), hout) for h, d in zip(hiddens[:2], drafts[:2])]
+        for i in range(3):
+            fv.run_host(hargs[i % 2], raw)
+        D.barrier(ranks)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            fv.run_host(hargs[i % 2], raw)
+        torch.cuda.synchronize()
+        e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
+        res["e2e"] = {"value": w.rows * ranks.world * e2e_steps / e2e_s, "unit": UNIT,
+                      "h2d_bytes_per_step": w.rows * w.hidden * 2 + w.B * w.K * 4,
+                      "d2h_bytes_per_step": w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12, "steps": e2e_steps,
+                      "api": "fly_verify_run_host (hidden states and drafts in pinned host buffers; weight resident)"}
+    if library:
+        # context only: the library GEMM (torch.matmul -> cuBLAS) on the SAME shape, writing bf16 logits, same
+        # number of back-to-back launches.  It does none of the verification; it shows what the shape allows.
+        lib_logits = torch.empty(w.rows, w.V, dtype=torch.bfloat16, device=device)
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                torch.matmul(hiddens[0], weight, out=lib_logits)
+            stream.synchronize()
+            l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            l0.record(stream)
+            for i in range(n):
+                torch.matmul(hiddens[i % nbuf], weight, out=lib_logits)
+            l1.record(stream)
+            stream.synchronize()
+        lib_ms = l0.elapsed_time(l1) / n
+        res["library_gemm_same_shape"] = {
+            "us_per_step": lib_ms * 1e3, "tflops": flops / (lib_ms * 1e-3) / 1e12,
+            "note": "torch.matmul (cuBLAS) hidden x weight -> bf16 logits only, no verification; context, "
+                    "timed after the main measurement"}
+        del lib_logits
+    res["weight"] = weight
+    fv.close()
+    return res
+
+
+def fused_row(w, r):
+    row = {"rows_per_step": w.rows, "flops_per_step": r["flops"], "steps": r["steps"], "us_per_step": r["ms"] * 1e3,
+           "positions_per_s": w.rows / (r["ms"] * 1e-3), "tflops": r["tflops"], "frac_of_burst": r["frac_of_burst"],
+           "frac_of_sustained": r["frac_of_sustained"], "clocks": r["clocks"]}
+    if "library_gemm_same_shape" in r:
+        row["library_gemm_same_shape"] = r["library_gemm_same_shape"]
+    return row
+
+
+def run_fused(args, w):
+    import torch
+    from paper_2511_22972_b200 import dist as D
+    warmup = 5 if args.warmup is None else max(args.warmup, 3)
+    ranks = D.init_from_env("nccl")
+    assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
+    torch.cuda.set_device(ranks.local_rank)
+    device = torch.device("cuda", ranks.local_rank)
+    peaks = measured_peaks()
+    r = bench_fused(w, ranks, device, args.steps or 200, warmup, peaks)
+    rows_all = w.rows * ranks.world
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": rows_all / (r["ms"] * 1e-3), "unit": UNIT, "n_gpus": ranks.world, "steps": r["steps"],
+        "warmup": warmup, "ms_per_step": r["ms"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "hidden": w.hidden,
                    "theta_nats": w.theta, "W": w.W, "boundary": w.boundary, "parallelism": f"dp{ranks.world}",
                    "launch": "stream", "l2": f"the weight ({w.hidden * w.V * 2 / 1e9:.2f} GB, read once per step) is larger than L2"},
-        "tflops": achieved,
+        "tflops": r["tflops"],
         "roofline": {"bound": "tensor", "kernel": "lmhead_verify_kernel (tcgen05 GEMM + entropy/argmax epilogue)",
-                     "achieved": achieved, "peak": burst, "peak_kind": f"of {kind} (bf16 burst)", "unit": "TFLOP/s",
-                     "frac": achieved / burst, "frac_of_sustained": achieved / sustained, "flops_per_launch": flops,
-                     "us_per_launch": ms_per_step * 1e3,
-                     "note": "duration = whole step (GEMM kernel + acceptance-scan kernel, the latter ~3 us)",
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
-        "hbm_gbs": (w.hidden * w.V * 2 + w.rows * w.hidden * 2) / (ms_per_step * 1e-3) / 1e9,
-        "library_gemm_same_shape": {"ms_per_step": lib_ms, "tflops": flops / (lib_ms * 1e-3) / 1e12,
-                                    "note": "torch.matmul (cuBLAS) hidden x weight -> bf16 logits only, no verification; "
-                                            "context, timed after the main measurement"},
-        "e2e": {"value": rows_all * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                "api": "fly_verify_run_host (hidden states and drafts in pinned host buffers; weight resident)"},
-        "gpu_launches": launches_per_step * args.steps,
-        "clocks": clk.summary(),
+                     "achieved": r["tflops"], "peak": peaks["burst"], "peak_kind": f"of {peaks['kind']} (bf16 burst)",
+                     "unit": "TFLOP/s", "frac": r["tflops"] / peaks["burst"], "frac_of_sustained": r["frac_of_sustained"],
+                     "flops_per_launch": r["flops"], "us_per_launch": r["ms"] * 1e3,
+                     "note": "duration = whole step (GEMM kernel + fold + acceptance-scan kernels, the latter two ~3 us)",
+                     "traffic": ncu_traffic("lmhead_verify_kernel", w.V)},
+        "hbm_gbs": r["hbm_gbs"],
+        "library_gemm_same_shape": r["library_gemm_same_shape"],
+        "e2e": r["e2e"],
+        "gpu_launches": r["launches_per_step"] * r["steps"],
+        "clocks": r["clocks"],
     }
     if ranks.is_main and ranks.world == 1 and not args.no_cpu_baseline:
-        wc = weight.cpu()
+        wc = r["weight"].cpu()
         t, rows = fused_oracle_sample(w, wc, 1, 0)
         line["cpu_baseline"] = {"value": rows / t, "unit": UNIT, "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                                 "sample": f"1 of {w.B} sequences ({rows} rows, all V={w.V}): fp64 matmul (BLAS threads) + verification (1 thread)"}
     if ranks.is_main:
         print(json.dumps(line), flush=True)
-    fv.close()
     D.finalize(ranks)
 
+
+# ------------------------------------------------------------------------------------------------------
+# vocabulary-parallel mode
+# ------------------------------------------------------------------------------------------------------
+
+def run_vocab_parallel(args, w):
+    """--shard vocab: a tensor-parallel LM head leaves every rank with one slice of the vocabulary.  Per step
+    every rank reduces its slice to one 16-byte state per row (fly_verify_reduce_shard), the states are
+    all-gathered (one NCCL call; world 1: none) and every rank applies the rule (fly_verify_run_partials)."""
+    import torch
+    from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, dist as D, synthetic as S
+    warmup = 10 if args.warmup is None else max(args.warmup, 3)
+    if args.gpus > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")           # the communicator log shows the ranks and NVLS
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    ranks = D.init_from_env("nccl")
+    assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
+    torch.cuda.set_device(ranks.local_rank)
+    device = torch.device("cuda", ranks.local_rank)
+    peaks = measured_peaks()
+    off, width = D.shard_vocab(w.V, ranks)
+    ws = S.shrink(w, V=width)                                 # this rank's slice, drawn with the workload's recipe
+    slice_bytes = w.rows * width * w.elem_bytes
+    nbuf = max(2, -(-int(2.4 * L2_BYTES) // slice_bytes))
+    slices = [S.make_logits(ws, 1000 * ranks.rank + i, device=device).view(w.rows, width) for i in range(nbuf)]
+    draft = torch.randint(0, w.V, (w.B, w.K), device=device, dtype=torch.int32)
+    out = VerifyBuffers(w.B, w.K, device)
+    shard = FlyVerify(w.B, w.K, width, w.dtype, device=ranks.local_rank)
+    merge = FlyVerify(w.B, w.K, w.V, w.dtype, device=ranks.local_rank)
+    mine = torch.empty(w.rows, 4, dtype=torch.float32, device=device)
+    margs = merge.make_args(w.B, w.K, draft, out.accept_len, out.out_tokens, theta=w.theta, W=w.W, state_out=out.state,
+                            rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
+                            row_flags=out.row_flags)
+    stream = torch.cuda.Stream(device=device)
+    raw = stream.cuda_stream
+
+    def step(i):
+        shard.reduce_shard(slices[i], off, mine, raw)
+        allp = D.all_gather_partials(ranks, mine)
+        merge.run_partials(margs, allp, ranks.world, w.V, raw)
+
+    n = steps_for(max(slice_bytes / (peaks["hbm"] * 1e9), 10e-6), args.steps)
+    with ClockSampler(ranks.local_rank) as clk:
+        ms = time_calls(step, nbuf, stream, n, warmup, ranks, "stream") / n
+    value = w.rows / (ms * 1e-3)
+    achieved = slice_bytes / (ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": n, "warmup": warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "K": w.K, "V": w.V, "V_per_gpu": width, "logits_dtype": w.dtype,
+                   "theta_nats": w.theta, "W": w.W, "boundary": "reject", "parallelism": f"tp{ranks.world}",
+                   "launch": "stream", "collective": "all-gather of 16 bytes per row and rank" if ranks.world > 1 else "none (one rank)",
+                   "l2": f"slices rotate over {nbuf} distinct buffers = {nbuf * slice_bytes / 1e6:.0f} MB per GPU (> 2x L2)"},
+        "roofline": {"bound": "hbm", "kernel": "reduce_rows_flat (this rank's vocabulary slice)", "achieved": achieved,
+                     "peak": peaks["hbm"], "peak_kind": f"of {peaks['kind']}", "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                     "bytes_per_launch": slice_bytes, "us_per_launch": ms * 1e3,
+                     "note": "duration = whole step: slice reduction + fold + all-gather + merge + acceptance scan",
+                     "traffic": ncu_traffic("reduce_rows_flat", w.rows * width)},
+        "e2e": None,
+        "gpu_launches": 4 * n,
+        "clocks": clk.summary(),
+    }
+    if ranks.is_main:
+        print(json.dumps(line), flush=True)
+    shard.close()
+    merge.close()
+    D.finalize(ranks)
+
+
+# ------------------------------------------------------------------------------------------------------
+# reference arm (the oracle)
+# ------------------------------------------------------------------------------------------------------
 
 def run_reference_fused(args, w):
     rank = int(os.environ.get("RANK", "0"))
@@ -361,44 +641,37 @@ def run_reference_fused(args, w):
 
 
 def run_reference(args, w):
-    """--impl reference: the oracle on the host cores; rank 0 only."""
+    """--impl reference: the oracle on the host cores; rank 0 only.  Each step is a bounded sample of the
+    workload: a few sequences per core, all cores at once."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-    import torch
-    from oracle import fly_oracle as O
-    from paper_2511_22972_b200 import synthetic as S
-    torch.set_num_threads(1)
-    B = max(1, min(w.B, 48 // (w.K + 1)))          # bounded sample of the workload per step
-    ws = S.shrink(w, B=B)
-
-    def one(step):
-        logits = S.make_logits(ws, step, device="cpu")
-        draft = S.make_draft(ws, step, S.rank5(logits.view(-1, ws.V)))
-        return logits.double().numpy(), draft.numpy()
-
-    data = [one(i) for i in range(min(4, args.steps + args.warmup))]
-    st = np.array([[0, 0, -1]] * ws.B) if w.boundary == "carry" else None
-    for i in range(args.warmup):
-        O.verify_batch(*data[i % len(data)], w.theta, w.W, boundary=w.boundary, state_in=st)
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        O.verify_batch(*data[i % len(data)], w.theta, w.W, boundary=w.boundary, state_in=st)
-    dt = time.perf_counter() - t0
-    value = ws.rows * args.steps / dt
-    sample = f"each step = {ws.B} of {w.B} sequences ({ws.rows} rows x V={ws.V})"
+    op = OraclePool(w, rows_per_core=24)
+    try:
+        for i in range(args.warmup):
+            op.round(10 ** 6 + i)
+        dt = sum(op.round(i) for i in range(args.steps))
+    finally:
+        op.close()
+    value = op.rows_per_round * args.steps / dt
+    sample = "each step = " + op.sample(1).split(" of ", 1)[1]
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype, "theta_nats": w.theta,
                    "W": w.W, "boundary": w.boundary, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": op.workers, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------------
+
+EXTRA_WORKLOADS = ("tiny_verify", "llama3_vocab_batch", "long_draft_batch", "high_batch_serving",
+                   "paper_default_70b", "paper_default_405b", "fused_lm_head")
 
 
 def main():
@@ -408,9 +681,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="llama3_vocab_batch")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--launch", default="stream", choices=["stream", "graph"])
-    ap.add_argument("--no-overlap", action="store_true",
-                    help="plain stream order between steps (no programmatic dependent launch)")
+    ap.add_argument("--launch", default="graph", choices=["stream", "graph"],
+                    help="logits path: launch the timed steps from CUDA graphs (default) or one by one from the host")
+    ap.add_argument("--shard", default="batch", choices=["batch", "vocab"])
+    ap.add_argument("--no-extra", action="store_true", help="time only --workload (no `workloads` object)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--vocab", type=int, default=None, help="run the workload's recipe at another vocabulary size "
                     "(smaller cases for profiler captures); recorded in config")
@@ -429,102 +703,81 @@ def main():
     if w.hidden:
         run_fused(args, w)
         return
-    # ~0.15 s of timed work by default: long enough for a dozen clock samples, short enough to be timed in the
-    # same regime as the copy that the HBM peak was measured with (a burst, best of 10)
-    args.steps = args.steps or min(200000, max(2000, int(0.15 / (w.rows * w.V * w.elem_bytes / 6.0e12))))
-    args.warmup = 20 if args.warmup is None else max(args.warmup, 3)
+    if args.shard == "vocab":
+        run_vocab_parallel(args, w)
+        return
+    warmup = 20 if args.warmup is None else max(args.warmup, 3)
 
     import torch
-    from paper_2511_22972_b200 import FlyVerify, VerifyBuffers, dist as D
+    from paper_2511_22972_b200 import dist as D
     ranks = D.init_from_env("nccl")
     assert ranks.world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={ranks.world}"
     torch.cuda.set_device(ranks.local_rank)
     device = torch.device("cuda", ranks.local_rank)
-    overlap = not args.no_overlap
+    peaks = measured_peaks()
 
-    step_bytes = w.rows * w.V * w.elem_bytes
-    nbuf = max(2, -(-int(2.4 * L2_BYTES) // step_bytes))     # rotate over > 2x L2 of distinct inputs
-    bufs = build_inputs(w, device, nbuf)
-    out = VerifyBuffers(w.B, w.K, device)
-    fv = FlyVerify(w.B, w.K, w.V, w.dtype, device=ranks.local_rank)
-    fv.set_stream_overlap(overlap)
-    carry = w.boundary == "carry"
-    arglist = [fv.make_args(w.B, w.K, d, out.accept_len, out.out_tokens, logits=l, theta=w.theta, W=w.W,
-                            boundary=w.boundary, state_in=out.state if carry else None, state_out=out.state,
-                            rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
-                            row_flags=out.row_flags) for (l, d) in bufs]
-    stream = torch.cuda.Stream(device=device)
-
-    # ---- whole step, device-resident inputs --------------------------------------------------------
-    with ClockSampler(ranks.local_rank) as clk:
-        ms_total = time_steps(fv, arglist, stream, args.steps, args.warmup, ranks, args.launch)
-        launches_per_step = fv.last_launch_count
-    # The step is ONE launch (the acceptance scan is the tail of the row-reduction kernel), so the
-    # dominant kernel's average launch duration is the step time measured above.
-    assert launches_per_step == 1, launches_per_step
-    ms_reduce = ms_total
-    ms_per_step = ms_total / args.steps
+    # ---- the named workload: whole steps over device-resident inputs, serial and overlapped ---------------
+    r = bench_logits(w, ranks, device, args.steps, warmup, args.launch, peaks)
+    assert r["launches_per_step"] == 1, r["launches_per_step"]     # the acceptance scan is the tail of the reduction
+    ms_per_step = r["serial_ms"]
     rows_all = w.rows * ranks.world
     value = rows_all / (ms_per_step * 1e-3)
-
-    # ---- the same steps without cross-step overlap (plain stream order), for the record ---------------
-    fv.set_stream_overlap(False)
-    ms_serial = time_steps(fv, arglist, stream, max(args.steps // 4, 10), 3, ranks, args.launch) / max(args.steps // 4, 10)
-    fv.set_stream_overlap(overlap)
-
-    # ---- end to end through the host-buffer entry point ------------------------------------------------
-    e2e_steps = max(10, min(200, args.steps // 50))
-    host_l = [b[0].cpu().pin_memory() for b in bufs[:2]]
-    host_d = [b[1].cpu().pin_memory() for b in bufs[:2]]
-    hout = VerifyBuffers(w.B, w.K, device, pinned=True)
-    hargs = [fv.make_args(w.B, w.K, d, hout.accept_len, hout.out_tokens, logits=l, theta=w.theta, W=w.W,
-                          boundary=w.boundary, state_in=hout.state if carry else None, state_out=hout.state,
-                          rollback=hout.rollback, target_argmax=hout.target_argmax, entropy=hout.entropy,
-                          row_flags=hout.row_flags) for l, d in zip(host_l, host_d)]
-    raw = stream.cuda_stream
-    for i in range(3):
-        fv.run_host(hargs[i % 2], raw)
-    D.barrier(ranks)
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for i in range(e2e_steps):
-        fv.run_host(hargs[i % 2], raw)          # synchronises the stream before returning
-    torch.cuda.synchronize()
-    e2e_s = D.max_over_ranks(ranks, time.perf_counter() - t0)
-    h2d = step_bytes + w.B * w.K * 4 + (w.B * 12 if carry else 0)
-    d2h = w.B * 4 * 2 + w.rows * 4 * 4 + w.B * 12
-    e2e_value = rows_all * e2e_steps / e2e_s
-
-    peak, peak_kind = measured_hbm_peak()
-    achieved = step_bytes / (ms_reduce / args.steps * 1e-3) / 1e9
+    achieved = r["step_bytes"] / (ms_per_step * 1e-3) / 1e9
+    e2e = e2e_logits(w, r, ranks, device, r["steps"])
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks.world, "steps": r["steps"],
+        "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
                    "theta_nats": w.theta, "W": w.W, "boundary": w.boundary, "parallelism": f"dp{ranks.world}",
-                   "launch": args.launch, "stream_overlap": overlap,
-                   "l2": f"inputs rotate over {nbuf} distinct buffers = {nbuf * step_bytes / 1e6:.0f} MB (> 2x L2)"},
+                   "launch": args.launch, "order": "plain stream order (each step waits for the previous kernel before its first read)",
+                   "l2": f"inputs rotate over {r['nbuf']} distinct buffers = {r['nbuf'] * r['step_bytes'] / 1e6:.0f} MB (> 2x L2)"},
         "hbm_gbs": rows_all * w.V * w.elem_bytes / (ms_per_step * 1e-3) / 1e9,
-        "hbm_pct_of_peak": 100.0 * step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
-        "serialized": {"ms_per_step": ms_serial, "value": rows_all / (ms_serial * 1e-3),
-                       "note": "same steps in plain stream order (no overlap between consecutive steps)"},
-        "roofline": {"bound": "hbm", "kernel": "reduce_rows_vec (row reduction: entropy + argmax partial states)",
-                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": achieved / peak, "bytes_per_launch": step_bytes,
-                     "us_per_launch": ms_reduce / args.steps * 1e3,
-                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "steps": e2e_steps, "api": "fly_verify_run_host (pinned host buffers)"},
-        "gpu_launches": launches_per_step * args.steps,
-        "clocks": clk.summary(),
+        "hbm_pct_of_peak": 100.0 * achieved / peaks["hbm"],
+        "overlapped": {"ms_per_step": r["overlapped_ms"], "value": rows_all / (r["overlapped_ms"] * 1e-3),
+                       "frac": r["step_bytes"] / (r["overlapped_ms"] * 1e-3) / 1e9 / peaks["hbm"],
+                       "note": "same steps with inputs_ready: a step may read its logits while the previous step drains; "
+                               "valid only over inputs that are complete beforehand, not inside a decode loop"},
+        "roofline": {"bound": "hbm", "kernel": "reduce_rows_flat (row reduction + acceptance scan in its tail; one launch per step)",
+                     "achieved": achieved, "peak": peaks["hbm"], "peak_kind": f"of {peaks['kind']} (copy bandwidth)",
+                     "unit": "GB/s", "frac": achieved / peaks["hbm"], "bytes_per_launch": r["step_bytes"],
+                     "us_per_launch": ms_per_step * 1e3,
+                     "note": "one launch per step in plain stream order, so the step time is the launch duration plus "
+                             "the gap to the next launch",
+                     "frac_overlapped": r["step_bytes"] / (r["overlapped_ms"] * 1e-3) / 1e9 / peaks["hbm"],
+                     "traffic": ncu_traffic("reduce_rows_flat", w.rows * w.V * w.elem_bytes)},
+        "e2e": e2e,
+        "gpu_launches": r["launches_per_step"] * r["steps"],
+        "clocks": r["clocks"],
     }
+    main_row = logits_row(w, r, peaks, ranks.world)
+    long_enough = r["steps"] * r["serial_ms"] * 1e-3 >= MIN_TIMED_S
+    r["fv"].close()
+    del r
+
+    # ---- every other workload, same protocol (one GPU only: it is a report, not part of the scaling run) ----
+    if ranks.world == 1 and not args.no_extra and not (args.vocab or args.batch):
+        rows = {}
+        for name in EXTRA_WORKLOADS:
+            wx = S.WORKLOADS[name]
+            torch.cuda.empty_cache()
+            if name == w.name and long_enough:
+                rows[name] = main_row
+            elif wx.hidden:
+                rf = bench_fused(wx, ranks, device, None, 5, peaks, e2e=False)
+                rows[name] = fused_row(wx, rf)
+                del rf
+            else:
+                rx = bench_logits(wx, ranks, device, None, warmup, args.launch, peaks, near_miss=False)
+                rows[name] = logits_row(wx, rx, peaks, 1)
+                rx["fv"].close()
+                del rx
+        line["workloads"] = rows
     if ranks.is_main and ranks.world == 1 and not args.no_cpu_baseline:
         v, sample, cores = oracle_rate(w)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
     if ranks.is_main:
         print(json.dumps(line), flush=True)
-    fv.close()
     D.finalize(ranks)
 
 

@@ -16,7 +16,10 @@
  *     Position K+1 is the bonus position.
  *   - fly_verify_run is asynchronous on the given CUDA stream, allocates
  *     nothing and never synchronises the host with the device.
- *   - A handle is not thread-safe: use one per host thread, or serialise the calls on it.
+ *   - A handle owns one set of scratch buffers: steps issued through one handle
+ *     must run one after the other on the GPU (keep a handle on one stream at a
+ *     time) and the host calls on it must not overlap (one host thread at a
+ *     time).  Use one handle per stream.
  *   - No function throws, aborts or traps.  Misuse that the host can see is
  *     reported by the return code before anything is launched; conditions that
  *     depend on device data (non-finite logits, draft ids out of range) are
@@ -133,6 +136,24 @@ typedef struct {
    * the given tokens replace the argmax in the match indicator (Eq. 2) and in the emitted tokens;
    * the entropy gate still uses the entropy of the logits.  target_argmax still reports the argmax. */
   const int32_t* target_tokens;
+
+  /* Temperature T of the target distribution: the entropy of Eq. 5 is taken of softmax(l / T), the
+   * distribution a caller that samples at temperature T draws from (the paper reports temperature-1
+   * results next to the greedy ones).  0 means 1 (the logits as they are); otherwise 1e-6 <= T <= 1e6.
+   * 1/T is folded into the constant that turns a logit into a base-2 exponent, so it costs nothing.  The
+   * greedy token (Eq. 1) does not depend on T. */
+  double temperature;
+
+  /* Launch ordering of the logits path.  The row reduction is always launched so that it may be
+   * scheduled while the previous kernel in the stream drains (programmatic dependent launch).
+   * 0 (default): plain stream order.  The kernel waits for the previous kernel to complete before its
+   *    first read; only its launch latency is hidden.  Always correct.
+   * 1: the caller guarantees that the logits and draft tokens of this step were complete BEFORE the
+   *    previous kernel in the stream was launched (e.g. a queue of steps over inputs that are already in
+   *    memory).  The kernel then starts READING at once, next to the draining previous kernel, and waits
+   *    only before its first write.  Wrong results if the guarantee does not hold - in a decode loop, where
+   *    the previous kernel produces this step's logits, leave it 0. */
+  int32_t inputs_ready;
 } fly_verify_args_t;
 
 /* Runs one verification step on `cuda_stream` (a cudaStream_t; NULL = default
@@ -153,7 +174,8 @@ fly_status_t fly_verify_run_host(fly_verify_t* handle, const fly_verify_args_t* 
  * (Section 3, implementation details); with a tensor-parallel LM head every GPU holds the logits of
  * one slice of the vocabulary only.  Eq. 1 and Eq. 5 then split into a per-slice reduction and a
  * merge: for a slice with maximum m_k, S_k = sum 2^(z - r_k) and u_k = sum 2^(z - r_k)(z - r_k)
- * (z = logit * log2 e, r_k = m_k * log2 e), the whole row has m = max m_k,
+ * (z = logit * log2 e / T, r_k = m_k * log2 e / T, T = the temperature, which every rank and the merging
+ * call must pass alike; 0 = 1), the whole row has m = max m_k,
  * S = sum_k 2^(r_k - r) S_k, u = sum_k 2^(r_k - r)(u_k + (r_k - r) S_k), entropy
  * H = ln2 (log2 S - u / S), and the greedy token is the index of the largest m_k (lowest index on
  * ties).  One state per row and rank (16 bytes) is all that has to cross the interconnect.
@@ -174,7 +196,8 @@ typedef struct {
   int32_t argmax;   /* global token id of the first entry equal to m_k */
 } fly_partial_t;
 fly_status_t fly_verify_reduce_shard(fly_verify_t* handle, int32_t rows, const void* logits, int64_t row_stride,
-                                     int32_t vocab_offset, fly_partial_t* partial_out, void* cuda_stream);
+                                     int32_t vocab_offset, double temperature, fly_partial_t* partial_out,
+                                     void* cuda_stream);
 fly_status_t fly_verify_run_partials(fly_verify_t* handle, const fly_verify_args_t* args, const fly_partial_t* partials,
                                      int32_t world, int32_t total_vocab, void* cuda_stream);
 
@@ -213,8 +236,8 @@ fly_status_t fly_pld_draft(int32_t device, int32_t B, const int32_t* tokens, int
  *                                 weight must be NULL); inputs and outputs are still the caller's
  *
  * Limits: B <= FLY_STATIC_MAX_BATCH, K <= 63 and B*(K+1) <= FLY_STATIC_MAX_PIECES.  Rows are cut into
- * pieces as usual, but never into more than FLY_STATIC_MAX_PIECES pieces in total.  A step beyond the
- * limits returns FLY_ERR_TOO_LARGE and launches nothing.
+ * pieces as usual, but the partial-state slots of all rows together never exceed FLY_STATIC_MAX_PIECES.
+ * A step beyond the limits returns FLY_ERR_TOO_LARGE and launches nothing.
  *
  * The first call on each device looks up the device address of the built-in
  * array (which also makes the CUDA runtime load the library's device code).
@@ -236,24 +259,21 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
 /* Options of a handle (fly_verify_set_option).  None of them changes results
  * beyond fp32 rounding order.
  *
- * FLY_OPT_SPLITS          > 0 forces every row to be cut into that many pieces (1..32), each reduced
- *                         by its own thread block; 0 (default) chooses from the shape.
+ * FLY_OPT_SPLITS          The row reduction gives every thread block the same number of bytes and sizes the grid
+ *                         to fill the device once.  0 (default): small steps cut every row into the same number
+ *                         of whole pieces (at least 16 KB each); large steps lay the rows end to end and cut
+ *                         that range evenly, so a block may cover the end of one row and the start of the next.
+ *                         s > 0: every row is cut into exactly s pieces (1..32), one thread block each (for
+ *                         tests and experiments).
  * FLY_OPT_SCAN_MODE       0 (default): the acceptance scan runs as the tail of the row-reduction
- *                         kernel (the last block to finish a sequence's rows verifies it; one launch
+ *                         kernel (the block that completes a sequence's rows verifies it; one launch
  *                         per step).  1: it runs as a kernel of its own (two launches per step).
- * FLY_OPT_STREAM_OVERLAP  1: the row reduction is launched as a programmatic dependent of the
- *                         previous kernel in the stream: it may start READING its logits while that
- *                         kernel is still draining and waits for it to complete only before its
- *                         first write.  Only correct if the logits of this step were complete
- *                         before that previous kernel started (e.g. back-to-back steps over inputs
- *                         already in memory).  0 (default): plain stream order.
  * FLY_OPT_WEIGHT_LAYOUT   fused path only.  0 (default): weight is [hidden, V] row-major (V contiguous).
  *                         1: weight is [V, hidden] row-major (hidden contiguous), the layout in which
  *                         linear layers are usually stored. */
 typedef enum {
   FLY_OPT_SPLITS = 0,
   FLY_OPT_SCAN_MODE = 1,
-  FLY_OPT_STREAM_OVERLAP = 2,
   FLY_OPT_WEIGHT_LAYOUT = 3
 } fly_option_t;
 fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, int32_t value);
@@ -271,11 +291,25 @@ fly_status_t fly_verify_device_status(fly_verify_t* handle, void* cuda_stream);
  * next fly_verify_device_status reports FLY_ERR_TIMEOUT.  Nothing faults or hangs. */
 fly_status_t fly_verify_selftest_wait(fly_verify_t* handle, void* cuda_stream);
 
-/* Introspection, host only (no CUDA call): the number of pieces into which the logits path cuts every
- * row of row_bytes bytes when `rows` rows are reduced on a device with sm_count SMs, with or without
- * FLY_OPT_STREAM_OVERLAP.  1..32; 0 for invalid arguments.  (Rows shorter than 32 segments of 16 bytes
- * and unaligned rows may get fewer pieces than this at run time.) */
-int32_t fly_verify_plan_splits(int32_t sm_count, int64_t rows, int64_t row_bytes, int32_t stream_overlap);
+/* Introspection, host only (no CUDA call): the launch geometry the logits path chooses for `rows` rows of
+ * `vocab` logits of `dtype` on a device with sm_count SMs.  vector_path = 1 if base, row stride and row length
+ * allow 16-byte loads (a unit is then a 16-byte segment, else one logit).  forced_pieces as FLY_OPT_SPLITS.
+ *   grid             thread blocks
+ *   units_per_block  block b reduces the flat unit range [b * units_per_block, (b + 1) * units_per_block)
+ *   units_per_row    whole units in a row
+ *   row_span         units a row takes in that flat range (>= units_per_row; equal when rows are packed
+ *                    end to end, a multiple of units_per_block when rows are cut into whole pieces)
+ *   slots            partial-state slots reserved per row (>= the pieces of any row)
+ * Returns FLY_ERR_INVALID_ARG for sizes out of range. */
+typedef struct {
+  int32_t grid;
+  int32_t slots;
+  int64_t units_per_block;
+  int64_t units_per_row;
+  int64_t row_span;
+} fly_plan_t;
+fly_status_t fly_verify_plan(int32_t sm_count, int64_t rows, int32_t vocab, fly_dtype_t dtype, int32_t vector_path,
+                             int32_t inputs_ready, int32_t forced_pieces, fly_plan_t* out);
 
 /* Number of kernels the last fly_verify_run enqueued (for accounting). */
 int32_t fly_verify_last_launch_count(const fly_verify_t* handle);

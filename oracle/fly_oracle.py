@@ -308,7 +308,8 @@ class BatchResult(NamedTuple):
 def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
                  theta_unit: str = "nats", boundary: str = "reject",
                  state_in: Optional[np.ndarray] = None,
-                 target_tokens: Optional[np.ndarray] = None) -> BatchResult:
+                 target_tokens: Optional[np.ndarray] = None,
+                 temperature: float = 1.0) -> BatchResult:
     """One verification step.  logits [B, K+1, V] float64 (exactly widened
     input bits), draft [B, K] integer.  Entropy is computed for every row
     (the paper needs it only at mismatches; the extra rows change nothing).
@@ -317,8 +318,16 @@ def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
     target_tokens [B, K+1] (optional, an extension outside the paper's method text, which defines y_i
     only as the argmax of Eq. 1): tokens the caller drew from the target distributions.  They take the
     place of y_i in Eq. 2 and in the emitted tokens; the gate still uses the entropy of the logits and
-    target_argmax still reports the argmax.  An id outside [0, V) is flagged and never accepted."""
+    target_argmax still reports the argmax.  An id outside [0, V) is flagged and never accepted.
+
+    temperature T > 0 (an extension for the paper's temperature-1 result columns; its method text is
+    greedy): the distribution of Eq. 1 / Eq. 5 is softmax(l / T), i.e. the statistics are those of the
+    logits divided by T.  Dividing by a positive number keeps the order, so y_i is unchanged."""
     logits = np.asarray(logits, dtype=np.float64)
+    if not (temperature > 0.0):
+        raise ValueError("temperature must be positive")
+    if temperature != 1.0:
+        logits = logits / float(temperature)
     B, K1, V = logits.shape
     K = K1 - 1
     draft = np.asarray(draft).reshape(B, K)

@@ -17,12 +17,12 @@ FLY_STATIC_MAX_BATCH, FLY_STATIC_MAX_PIECES = 1024, 16384
 FLY_F32, FLY_BF16 = 0, 1
 FLY_THETA_NATS, FLY_THETA_NORMALIZED = 0, 1
 FLY_BOUNDARY_REJECT, FLY_BOUNDARY_CARRY = 0, 1
-FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_STREAM_OVERLAP, FLY_OPT_WEIGHT_LAYOUT = range(4)
+FLY_OPT_SPLITS, FLY_OPT_SCAN_MODE, FLY_OPT_WEIGHT_LAYOUT = 0, 1, 3
 
 EXPORTS = (
     "fly_verify_create", "fly_verify_destroy", "fly_verify_run", "fly_verify_run_host", "fly_verify_run_static",
     "fly_verify_device_status", "fly_verify_selftest_wait", "fly_verify_reduce_shard", "fly_verify_run_partials",
-    "fly_pld_draft", "fly_verify_plan_splits",
+    "fly_pld_draft", "fly_verify_plan",
     "fly_verify_set_option", "fly_verify_last_launch_count", "fly_verify_last_cuda_error",
     "fly_status_string",
 )
@@ -44,7 +44,13 @@ class fly_verify_args_t(C.Structure):
         ("accept_len", C.c_void_p), ("rollback", C.c_void_p), ("out_tokens", C.c_void_p),
         ("target_argmax", C.c_void_p), ("entropy", C.c_void_p), ("row_flags", C.c_void_p),
         ("target_tokens", C.c_void_p),
+        ("temperature", C.c_double), ("inputs_ready", C.c_int32),
     ]
+
+
+class fly_plan_t(C.Structure):
+    _fields_ = [("grid", C.c_int32), ("slots", C.c_int32), ("units_per_block", C.c_int64), ("units_per_row", C.c_int64),
+                ("row_span", C.c_int64)]
 
 
 class FlyError(RuntimeError):
@@ -81,7 +87,8 @@ def lib() -> C.CDLL:
     L.fly_verify_device_status.restype = C.c_int
     L.fly_verify_selftest_wait.argtypes = [C.c_void_p, C.c_void_p]
     L.fly_verify_selftest_wait.restype = C.c_int
-    L.fly_verify_reduce_shard.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
+    L.fly_verify_reduce_shard.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int64, C.c_int32, C.c_double, C.c_void_p,
+                                          C.c_void_p]
     L.fly_verify_reduce_shard.restype = C.c_int
     L.fly_verify_run_partials.argtypes = [C.c_void_p, C.POINTER(fly_verify_args_t), C.c_void_p, C.c_int32, C.c_int32,
                                           C.c_void_p]
@@ -89,8 +96,9 @@ def lib() -> C.CDLL:
     L.fly_pld_draft.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.fly_pld_draft.restype = C.c_int
-    L.fly_verify_plan_splits.argtypes = [C.c_int32, C.c_int64, C.c_int64, C.c_int32]
-    L.fly_verify_plan_splits.restype = C.c_int32
+    L.fly_verify_plan.argtypes = [C.c_int32, C.c_int64, C.c_int32, C.c_int, C.c_int32, C.c_int32, C.c_int32,
+                                  C.POINTER(fly_plan_t)]
+    L.fly_verify_plan.restype = C.c_int
     L.fly_verify_set_option.argtypes = [C.c_void_p, C.c_int, C.c_int32]
     L.fly_verify_set_option.restype = C.c_int
     L.fly_verify_last_launch_count.argtypes = [C.c_void_p]
@@ -160,20 +168,17 @@ class FlyVerify:
         self.set_option(FLY_OPT_WEIGHT_LAYOUT, 1 if vocab_major else 0)
         self.weight_vd = bool(vocab_major)
 
-    def set_stream_overlap(self, on: bool):
-        self.set_option(FLY_OPT_STREAM_OVERLAP, 1 if on else 0)
-
     def device_status(self, stream: int = 0) -> int:
         """fly_verify_device_status: synchronises the stream; FLY_OK or FLY_ERR_TIMEOUT."""
         return int(lib().fly_verify_device_status(self._h, C.c_void_p(stream)))
 
-    def reduce_shard(self, logits, vocab_offset: int, partial_out, stream: int = 0):
+    def reduce_shard(self, logits, vocab_offset: int, partial_out, stream: int = 0, temperature: float = 0.0):
         """fly_verify_reduce_shard: logits [rows, vocab_slice] (a strided view is fine) -> partial_out
         [rows, 4] (any 16-byte element type, e.g. float32 x 4)."""
         rows = logits.shape[0]
         assert logits.shape[1] == self.vocab and logits.stride(1) == 1
         st = lib().fly_verify_reduce_shard(self._h, int(rows), _ptr(logits), int(logits.stride(0)), int(vocab_offset),
-                                           _ptr(partial_out), C.c_void_p(stream))
+                                           float(temperature), _ptr(partial_out), C.c_void_p(stream))
         if st != FLY_OK:
             raise FlyError(st, "fly_verify_reduce_shard", lib().fly_verify_last_cuda_error(self._h))
 
@@ -195,7 +200,7 @@ class FlyVerify:
     def make_args(self, B, K, draft, accept_len, out_tokens, logits=None, row_stride=0, hidden=None,
                   weight=None, theta=1.0, theta_unit="nats", W=3, boundary="reject", state_in=None,
                   state_out=None, rollback=None, target_argmax=None, entropy=None, row_flags=None,
-                  target_tokens=None):
+                  target_tokens=None, temperature=0.0, inputs_ready=False):
         a = fly_verify_args_t()
         a.B, a.K = int(B), int(K)
         a.logits, a.row_stride = _ptr(logits), int(row_stride)
@@ -209,6 +214,8 @@ class FlyVerify:
         a.accept_len, a.rollback, a.out_tokens = _ptr(accept_len), _ptr(rollback), _ptr(out_tokens)
         a.target_argmax, a.entropy, a.row_flags = _ptr(target_argmax), _ptr(entropy), _ptr(row_flags)
         a.target_tokens = _ptr(target_tokens)
+        a.temperature = float(temperature)
+        a.inputs_ready = 1 if inputs_ready else 0
         return a
 
     def run(self, args: fly_verify_args_t, stream: int = 0):
@@ -273,8 +280,19 @@ class VerifyBuffers:
         self.state = zero.pin_memory() if pinned else zero.to(device)
 
 
+def plan(sm_count: int, rows: int, vocab: int, dtype: str = "bf16", vector_path: bool = True, inputs_ready: bool = False,
+         forced_pieces: int = 0) -> fly_plan_t:
+    """fly_verify_plan: the launch geometry of the row reduction (host arithmetic only, no CUDA call)."""
+    out = fly_plan_t()
+    st = lib().fly_verify_plan(int(sm_count), int(rows), int(vocab), FLY_BF16 if dtype == "bf16" else FLY_F32,
+                               1 if vector_path else 0, 1 if inputs_ready else 0, int(forced_pieces), C.byref(out))
+    if st != FLY_OK:
+        raise FlyError(st, "fly_verify_plan")
+    return out
+
+
 def verify(fv: FlyVerify, logits, draft, out: VerifyBuffers, theta=1.0, W=3, theta_unit="nats",
-           boundary="reject", stream: int = 0, host: bool = False):
+           boundary="reject", stream: int = 0, host: bool = False, temperature=0.0, inputs_ready=False):
     """One verification step on logits [B, K+1, V] and draft [B, K] (int32).
     In carry mode out.state is both the carried-in and the carried-out state."""
     B, K1, V = logits.shape
@@ -283,13 +301,14 @@ def verify(fv: FlyVerify, logits, draft, out: VerifyBuffers, theta=1.0, W=3, the
     a = fv.make_args(B, K1 - 1, draft, out.accept_len, out.out_tokens, logits=logits,
                      row_stride=logits.stride(1), theta=theta, theta_unit=theta_unit, W=W, boundary=boundary,
                      state_in=out.state if carry else None, state_out=out.state, rollback=out.rollback,
-                     target_argmax=out.target_argmax, entropy=out.entropy, row_flags=out.row_flags)
+                     target_argmax=out.target_argmax, entropy=out.entropy, row_flags=out.row_flags,
+                     temperature=temperature, inputs_ready=inputs_ready)
     (fv.run_host if host else fv.run)(a, stream)
     return out
 
 
 def verify_fused(fv: FlyVerify, hidden, weight, draft, out: VerifyBuffers, theta=1.0, W=3, theta_unit="nats",
-                 boundary="reject", stream: int = 0, host: bool = False):
+                 boundary="reject", stream: int = 0, host: bool = False, temperature=0.0):
     """One verification step on the fused LM-head path: hidden [B*(K+1), D] bf16 and weight [D, V] bf16
     (device; with host=True hidden, draft and the outputs are host buffers, the weight stays on the device).
     The logits hidden @ weight are formed and reduced inside the kernel and never stored."""
@@ -302,6 +321,6 @@ def verify_fused(fv: FlyVerify, hidden, weight, draft, out: VerifyBuffers, theta
     a = fv.make_args(B, K, draft, out.accept_len, out.out_tokens, hidden=hidden, weight=weight, theta=theta,
                      theta_unit=theta_unit, W=W, boundary=boundary, state_in=out.state if carry else None,
                      state_out=out.state, rollback=out.rollback, target_argmax=out.target_argmax,
-                     entropy=out.entropy, row_flags=out.row_flags)
+                     entropy=out.entropy, row_flags=out.row_flags, temperature=temperature)
     (fv.run_host if host else fv.run)(a, stream)
     return out

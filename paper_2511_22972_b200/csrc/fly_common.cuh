@@ -23,7 +23,7 @@ constexpr uint32_t kFlagBadTarget = 4u;
 
 // Running state of one (piece of a) row in the base-2 domain.
 //   mx   largest logit seen (raw value; decides the argmax)
-//   S    sum 2^(z - r)            z = logit * log2(e),  r = mx * log2(e)
+//   S    sum 2^(z - r)            z = logit * scale,  r = mx * scale,  scale = log2(e) / temperature
 //   u    sum 2^(z - r) * (z - r)
 //   idx  lowest index holding mx
 // Entropy in nats (numerator of Eq. 5):  H = ln2 * (log2 S - u / S), for any
@@ -59,8 +59,8 @@ __device__ __forceinline__ uint32_t warp_min_u32(uint32_t v) { return __reduce_m
 
 // Rebase identity: sum 2^(z-r')(z-r') = 2^(r-r') * (u + (r-r') S).
 // Merges b into a; on equal maxima the lower index wins (Eq. 1 tie rule).
-__device__ __forceinline__ void merge_partial(Partial& a, const Partial& b) {
-  const float ra = a.mx * kLog2e, rb = b.mx * kLog2e;
+__device__ __forceinline__ void merge_partial(Partial& a, const Partial& b, float scale) {
+  const float ra = a.mx * scale, rb = b.mx * scale;
   const float r = fmaxf(ra, rb);
   const float da = ra - r, db = rb - r;  // <= 0, finite (mx is clamped to the mask floor)
   const float ea = ex2_approx(da), eb = ex2_approx(db);

@@ -19,11 +19,11 @@
 
 namespace {
 
-constexpr int kMaxSplits = 32;
-// 16-byte loads in flight per lane and slice in the row-reduction kernel.  Measured: 2 and 8 are
-// slower than 4, and loading the next slice before folding the current one (two register sets)
-// changes nothing.
+constexpr int kMaxSplits = 32;   // Partial slots per row in a handle's scratch
+// 16-byte loads per lane and slice in the row-reduction kernel (a warp keeps two slices: one in flight,
+// one being folded).
 constexpr int kReduceUnroll = 4;
+constexpr int64_t kMinBlockBytes = 16384;   // a block that gets less than this is all fixed cost
 constexpr int kMaxK = 63;
 
 struct DeviceGuard {
@@ -50,8 +50,6 @@ struct fly_verify {
   unsigned int* tickets = nullptr;   // [max_batch], zero between launches
   int forced_splits = 0;
   int scan_mode = 0;   // 0: fused tail, 1: separate kernel
-  int overlap = 0;
-  int last_splits = 1;
   int last_launches = 0;
   int last_cuda_error = 0;
   // fused LM-head path (cfg.hidden > 0)
@@ -81,41 +79,61 @@ fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
   return FLY_ERR_CUDA;
 }
 
-// Pieces per row.  Every block pays a fixed price (pipeline fill, block merge,
-// arrival ticket), so pieces should be large; but a grid that runs alone needs
-// enough blocks to fill every SM several times over and to divide evenly among
-// the SMs.  Among the allowed counts take the smallest whose blocks-per-SM
-// balance is within 3% of the best one, once there are >= 3.5 blocks per SM.
-// With stream overlap consecutive grids share the SMs, a single grid need not
-// fill the machine, and whole rows (or a few large pieces) are fastest.
-int auto_splits(const fly_verify* h, int64_t rows, int64_t row_bytes, int64_t max_pieces) {
-  const int64_t sms = h->sm_count;
-  int64_t cap = row_bytes / 32768;  // keep >= 32 KB per block ...
-  if (cap < 1) cap = 1;
-  if (2 * rows * cap < sms && row_bytes / 16384 > cap) cap = row_bytes / 16384;  // ... 16 KB when the grid is far from filling the SMs
-  if (cap > kMaxSplits) cap = kMaxSplits;
-  if (cap > max_pieces) cap = max_pieces;
-  if (h->overlap) {
-    for (int64_t s = 1; s <= cap; ++s)
-      if (4 * rows * s >= sms) return (int)s;
-    return (int)cap;
+// Launch geometry of the row reduction (the flat partition described at the head of reduce_kernel.cuh).
+// The grid should be resident all at once and give every block the same number of bytes: blocks then
+// finish together, whatever the number of rows, and a grid that runs alone has no ragged last wave.
+//   gmax   blocks that fit on the device at once (half of them when consecutive steps are meant to
+//          overlap, so that two grids can be resident together)
+//   n      units per row, min_units: a block should not get less than this
+//   cap    Partial slots available per row (>= 1)
+struct FlatPlan {
+  int64_t Q = 1;      // units per block
+  int64_t span = 1;   // units a row takes in the flat index space
+  int grid = 1;
+  int slots = 1;
+};
+// stride_units: units one thread block covers per loop iteration (all its warps, one slice each).
+FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int64_t stride_units, int cap,
+                   bool inputs_ready, int forced) {
+  FlatPlan pl;
+  const int bps = inputs_ready ? fly::kReduceBlocksPerSM / 2 : fly::kReduceBlocksPerSM;
+  const int64_t gmax = (int64_t)sm_count * (bps > 0 ? bps : 1);
+  int64_t s = 0;  // > 0: every row is cut into exactly s pieces
+  if (cap < 2) {
+    s = 1;        // one slot per row: whole rows
+  } else if (forced > 0) {
+    s = forced < cap ? forced : cap;
+  } else {
+    int64_t G = (rows * n + min_units - 1) / min_units;
+    if (G > gmax) G = gmax;
+    if (G < 1) G = 1;
+    const int64_t Qf = (rows * n + G - 1) / G;
+    if (rows <= gmax && Qf < 8 * stride_units) {
+      // Small step: a block has only a few slices per warp, and a row boundary inside it would add one.
+      // Cut rows into whole pieces instead, as many as still fit on the device at once.
+      s = gmax / rows;
+      if (s > n / min_units) s = n / min_units;
+      if (s > cap) s = cap;
+      if (s < 1) s = 1;
+    } else {
+      pl.Q = (Qf + 63) / 64 * 64;  // piece starts on 1 KB boundaries of the row where the row length allows
+      const int64_t qmin = (n + (cap - 1) - 1) / (cap - 1);  // a row never spans more than cap blocks
+      if (pl.Q < qmin) pl.Q = qmin;
+      pl.span = n;
+    }
   }
-  double best = 0.0;
-  int64_t first_full = 0;
-  for (int64_t s = 1; s <= cap; ++s) {
-    const int64_t n = rows * s;
-    if (2 * n < 7 * sms) continue;
-    if (!first_full) first_full = s;
-    const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
-    if (bal > best) best = bal;
+  if (s > 0) {
+    if (s > n) s = n;
+    pl.Q = (n + s - 1) / s;
+    if (s > 1) pl.Q = (pl.Q + 7) / 8 * 8;        // pieces start on 128-byte boundaries of the row
+    s = (n + pl.Q - 1) / pl.Q;                   // pieces that are not empty
+    pl.span = s * pl.Q;
   }
-  if (!first_full) return (int)cap;  // small problem: as many blocks as allowed
-  for (int64_t s = first_full; s <= cap; ++s) {
-    const int64_t n = rows * s;
-    const double bal = (double)n / (double)(sms * ((n + sms - 1) / sms));
-    if (bal >= best - 0.03) return (int)s;
-  }
-  return (int)cap;
+  const int64_t total = rows * pl.span;
+  pl.grid = (int)((total + pl.Q - 1) / pl.Q);
+  const int64_t most = s > 0 ? s : (n + pl.Q - 1) / pl.Q + 1;
+  pl.slots = (int)(most < cap ? most : cap);
+  return pl;
 }
 
 void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned grid, unsigned block, cudaStream_t st,
@@ -132,37 +150,58 @@ void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned gr
 }
 
 template <typename T>
-cudaError_t launch_reduce(const fly_verify* h, const void* logits, int64_t row_stride, int V, int64_t rows,
-                          int forced, fly::Partial* partials, cudaStream_t st, int* splits_out,
-                          fly::ScanParams tail, bool overlap) {
+bool vector_path_ok(const void* logits, int64_t row_stride, int V) {
+  return ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
+         (V >= fly::Seg<T>::kElems * 32);
+}
+
+// Launches the row reduction.  `tail` carries the acceptance scan's arguments (tickets == NULL: no scan in
+// this launch); its geometry fields are filled in here and returned through it for a stand-alone scan.
+template <typename T>
+cudaError_t launch_reduce(int sm_count, const void* logits, int64_t row_stride, int V, int64_t rows, int forced, int cap,
+                          fly::Partial* partials, cudaStream_t st, fly::ScanParams* tail, float scale,
+                          bool inputs_ready) {
   constexpr int kE = fly::Seg<T>::kElems;
-  const bool vec = ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
-                   (V >= kE * 32);
-  const int64_t row_bytes = (int64_t)V * (int64_t)sizeof(T);
-  if (vec) {
-    const int nseg = V / kE;
-    int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, nseg);
-    if (splits > nseg) splits = nseg;
-    const int segs_per_split = (nseg + splits - 1) / splits;
-    *splits_out = splits;
-    tail.splits = splits;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fill_launch(&cfg, attr, (unsigned)(rows * splits), fly::kReduceThreads, st, overlap);
-    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_vec<T, kReduceUnroll>, static_cast<const T*>(logits), row_stride, V, nseg,
-                              splits, segs_per_split, partials, tail);
-  } else {
-    int splits = forced > 0 ? forced : auto_splits(h, rows, row_bytes, (V + 31) / 32);
-    if (splits > V) splits = V;
-    const int elems_per_split = (V + splits - 1) / splits;
-    *splits_out = splits;
-    tail.splits = splits;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fill_launch(&cfg, attr, (unsigned)(rows * splits), fly::kReduceThreads, st, overlap);
-    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_scalar<T, 4>, static_cast<const T*>(logits), row_stride, V, splits,
-                              elems_per_split, partials, tail);
-  }
+  const bool vec = vector_path_ok<T>(logits, row_stride, V);
+  const int64_t n = vec ? V / kE : V;
+  const int64_t min_units = vec ? kMinBlockBytes / 16 : kMinBlockBytes / (int64_t)sizeof(T);
+  const int64_t stride_units = (int64_t)fly::kReduceWarps * kReduceUnroll * 32;
+  const FlatPlan pl = plan_flat(sm_count, rows, n, min_units, stride_units, cap, inputs_ready, forced);
+  fly::ReducePlan g;
+  g.n = n; g.span = pl.span; g.Q = pl.Q; g.total = rows * pl.span; g.slots = pl.slots; g.V = V; g.row_stride = row_stride;
+  g.scale = scale; g.wait_first = inputs_ready ? 0 : 1;
+  tail->splits = pl.slots;
+  tail->units_per_row = n;
+  tail->row_span = pl.span;
+  tail->Q = pl.Q;
+  tail->scale = scale;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fill_launch(&cfg, attr, (unsigned)pl.grid, fly::kReduceThreads, st, true);
+  // The rings of all resident blocks only fit on an SM whose L1/shared split favours shared memory.
+  constexpr int kRingBytes = fly::kReduceWarps * fly::kDepth * kReduceUnroll * 32 * 16;
+  static std::once_flag ring_once;
+  std::call_once(ring_once, [] {
+    cudaFuncSetAttribute(fly::reduce_rows_flat<T, kReduceUnroll, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    cudaFuncSetAttribute(fly::reduce_rows_flat<T, kReduceUnroll, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                         cudaSharedmemCarveoutMaxShared);
+    (void)cudaGetLastError();
+  });
+  cfg.dynamicSmemBytes = vec ? kRingBytes : 0;
+  if (vec)
+    return cudaLaunchKernelEx(&cfg, fly::reduce_rows_flat<T, kReduceUnroll, true>, static_cast<const T*>(logits), g, partials,
+                              *tail);
+  return cudaLaunchKernelEx(&cfg, fly::reduce_rows_flat<T, kReduceUnroll, false>, static_cast<const T*>(logits), g, partials,
+                            *tail);
+}
+
+cudaError_t launch_reduce_any(fly_dtype_t dt, int sm_count, const void* logits, int64_t row_stride, int V, int64_t rows,
+                              int forced, int cap, fly::Partial* partials, cudaStream_t st, fly::ScanParams* tail,
+                              float scale, bool inputs_ready) {
+  if (dt == FLY_BF16)
+    return launch_reduce<__nv_bfloat16>(sm_count, logits, row_stride, V, rows, forced, cap, partials, st, tail, scale,
+                                        inputs_ready);
+  return launch_reduce<float>(sm_count, logits, row_stride, V, rows, forced, cap, partials, st, tail, scale, inputs_ready);
 }
 
 cudaError_t launch_scan(const fly::ScanParams& p, cudaStream_t st) {
@@ -180,6 +219,8 @@ fly_status_t check_args(const fly_verify* h, const fly_verify_args_t* a) {
   if (a->W < 0) return FLY_ERR_INVALID_ARG;
   if (std::isnan(a->theta)) return FLY_ERR_INVALID_ARG;
   if (a->theta_unit != FLY_THETA_NATS && a->theta_unit != FLY_THETA_NORMALIZED) return FLY_ERR_INVALID_ARG;
+  if (!(a->temperature == 0.0 || (a->temperature >= 1e-6 && a->temperature <= 1e6))) return FLY_ERR_INVALID_ARG;
+  if (a->inputs_ready != 0 && a->inputs_ready != 1) return FLY_ERR_INVALID_ARG;
   if (a->boundary != FLY_BOUNDARY_REJECT && a->boundary != FLY_BOUNDARY_CARRY) return FLY_ERR_INVALID_ARG;
   const bool has_logits = a->logits != nullptr;
   const bool has_fused = a->hidden != nullptr || a->weight != nullptr;
@@ -193,6 +234,12 @@ fly_status_t check_args(const fly_verify* h, const fly_verify_args_t* a) {
     return FLY_ERR_INVALID_ARG;  // the paper's rule has no cross-round state
   }
   return FLY_OK;
+}
+
+// log2(e) / T: turns a logit into the base-2 exponent of its softmax weight at temperature T (0 = 1).
+float exponent_scale(double temperature) {
+  const double T = temperature == 0.0 ? 1.0 : temperature;
+  return (float)(1.4426950408889634 / T);
 }
 
 fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, const fly::Partial* partials, int splits);
@@ -242,6 +289,7 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     p.num_kb = (D + L::kBlockK - 1) / L::kBlockK;
     p.row0 = (int)row0;
     p.w_kmajor = h->weight_vd;
+    p.scale = exponent_scale(a->temperature);
     p.partials = h->lm_partials;
     p.status = h->lm_status;
     L::lmhead_verify_kernel<<<grid, L::kThreads, L::kSmemBytes, st>>>(h->map_w, h->map_h, p);
@@ -256,7 +304,7 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     const unsigned warps = fly::kFoldThreads / 32;
     fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, true);
     e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->lm_partials, grid, (int64_t)grid,
-                           (int64_t)1, h->lm_folded, (int)rows, 0);
+                           (int64_t)1, h->lm_folded, (int)rows, 0, exponent_scale(a->temperature), (int64_t)0, (int64_t)0);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
   }
@@ -276,6 +324,8 @@ float theta_to_nats(const fly_verify* h, const fly_verify_args_t* a) {
 fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, const fly::Partial* partials, int splits) {
   fly::ScanParams p;
   p.B = a->B; p.K = a->K; p.V = h->cfg.vocab; p.splits = splits;
+  p.units_per_row = 0; p.row_span = 0; p.Q = 0;  // every row has exactly `splits` parts unless the row reduction says otherwise
+  p.scale = exponent_scale(a->temperature);
   p.partials = partials;
   p.tickets = nullptr;
   p.draft = a->draft;
@@ -412,10 +462,6 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->scan_mode = v;
       return FLY_OK;
-    case FLY_OPT_STREAM_OVERLAP:
-      if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
-      h->overlap = v;
-      return FLY_OK;
     case FLY_OPT_WEIGHT_LAYOUT:
       if (v != 0 && v != 1) return FLY_ERR_INVALID_ARG;
       h->weight_vd = v;
@@ -426,9 +472,11 @@ fly_status_t fly_verify_set_option(fly_verify_t* h, fly_option_t opt, int32_t v)
 }
 
 fly_status_t fly_verify_reduce_shard(fly_verify_t* h, int32_t rows, const void* logits, int64_t row_stride,
-                                     int32_t vocab_offset, fly_partial_t* partial_out, void* cuda_stream) {
+                                     int32_t vocab_offset, double temperature, fly_partial_t* partial_out,
+                                     void* cuda_stream) {
   if (!h || !logits || !partial_out) return FLY_ERR_INVALID_ARG;
   if (rows < 1 || rows > h->max_rows || vocab_offset < 0) return FLY_ERR_INVALID_ARG;
+  if (!(temperature == 0.0 || (temperature >= 1e-6 && temperature <= 1e6))) return FLY_ERR_INVALID_ARG;
   const int V = h->cfg.vocab;
   if (row_stride != 0 && row_stride < V) return FLY_ERR_INVALID_ARG;
   if ((int64_t)vocab_offset + V > 0x7fffffff) return FLY_ERR_INVALID_ARG;
@@ -436,21 +484,19 @@ fly_status_t fly_verify_reduce_shard(fly_verify_t* h, int32_t rows, const void* 
   if (!g.ok) return FLY_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int64_t stride = row_stride ? row_stride : V;
+  const float scale = exponent_scale(temperature);
   fly::ScanParams none;
   memset(&none, 0, sizeof(none));  // tickets == NULL: no acceptance scan in this launch
-  int splits = 1;
-  cudaError_t e;
-  if (h->cfg.logits_dtype == FLY_BF16)
-    e = launch_reduce<__nv_bfloat16>(h, logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, none, false);
-  else
-    e = launch_reduce<float>(h, logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, none, false);
+  cudaError_t e = launch_reduce_any(h->cfg.logits_dtype, h->sm_count, logits, stride, V, rows, h->forced_splits, kMaxSplits,
+                                    h->partials, st, &none, scale, false);
   if (e != cudaSuccess) return cuda_fail(h, e);
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
   const unsigned warps = fly::kFoldThreads / 32;
   fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, true);
-  e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->partials, splits, (int64_t)splits, (int64_t)1,
-                         reinterpret_cast<fly::Partial*>(partial_out), (int)rows, (int)vocab_offset);
+  e = cudaLaunchKernelEx(&cfg, fly::fold_partials, (const fly::Partial*)h->partials, none.splits, (int64_t)none.splits,
+                         (int64_t)1, reinterpret_cast<fly::Partial*>(partial_out), (int)rows, (int)vocab_offset, scale,
+                         none.row_span, none.Q);
   if (e != cudaSuccess) return cuda_fail(h, e);
   h->last_launches = 2;
   return FLY_OK;
@@ -474,7 +520,8 @@ fly_status_t fly_verify_run_partials(fly_verify_t* h, const fly_verify_args_t* a
   fill_launch(&cfg, attr, (unsigned)((rows + warps - 1) / warps), fly::kFoldThreads, st, false);
   // all-gather layout: [world, rows]
   cudaError_t e = cudaLaunchKernelEx(&cfg, fly::fold_partials, reinterpret_cast<const fly::Partial*>(partials), (int)world,
-                                     (int64_t)1, (int64_t)rows, h->lm_folded, (int)rows, 0);
+                                     (int64_t)1, (int64_t)rows, h->lm_folded, (int)rows, 0, exponent_scale(a->temperature),
+                                     (int64_t)0, (int64_t)0);
   if (e != cudaSuccess) return cuda_fail(h, e);
   fly::ScanParams sp = scan_params(h, a, h->lm_folded, 1);
   sp.V = total_vocab;
@@ -530,12 +577,24 @@ fly_status_t fly_verify_selftest_wait(fly_verify_t* h, void* cuda_stream) {
   return e == cudaSuccess ? FLY_OK : cuda_fail(h, e);
 }
 
-int32_t fly_verify_plan_splits(int32_t sm_count, int64_t rows, int64_t row_bytes, int32_t stream_overlap) {
-  if (sm_count < 1 || rows < 1 || row_bytes < 1) return 0;
-  fly_verify h;
-  h.sm_count = sm_count;
-  h.overlap = stream_overlap ? 1 : 0;
-  return auto_splits(&h, rows, row_bytes, kMaxSplits);
+fly_status_t fly_verify_plan(int32_t sm_count, int64_t rows, int32_t vocab, fly_dtype_t dtype, int32_t vector_path,
+                             int32_t inputs_ready, int32_t forced_pieces, fly_plan_t* out) {
+  if (!out || sm_count < 1 || rows < 1 || rows > (int64_t)1 << 24 || vocab < 1) return FLY_ERR_INVALID_ARG;
+  if (dtype != FLY_F32 && dtype != FLY_BF16) return FLY_ERR_INVALID_ARG;
+  if (forced_pieces < 0 || forced_pieces > kMaxSplits) return FLY_ERR_INVALID_ARG;
+  const int64_t esz = dtype == FLY_BF16 ? 2 : 4;
+  const int64_t per_seg = 16 / esz;
+  if (vector_path && vocab < per_seg * 32) return FLY_ERR_INVALID_ARG;
+  const int64_t n = vector_path ? vocab / per_seg : vocab;
+  const int64_t min_units = vector_path ? kMinBlockBytes / 16 : kMinBlockBytes / esz;
+  const FlatPlan pl = plan_flat(sm_count, rows, n, min_units, (int64_t)fly::kReduceWarps * kReduceUnroll * 32, kMaxSplits,
+                                inputs_ready != 0, forced_pieces);
+  out->grid = pl.grid;
+  out->slots = pl.slots;
+  out->units_per_block = pl.Q;
+  out->units_per_row = n;
+  out->row_span = pl.span;
+  return FLY_OK;
 }
 
 int32_t fly_verify_last_launch_count(const fly_verify_t* h) { return h ? h->last_launches : 0; }
@@ -554,25 +613,13 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   h->last_launches = 0;
   if (!a->logits) return run_fused(h, a, st);
 
-  fly::ScanParams p = scan_params(h, a, h->partials, h->last_splits);
-
+  fly::ScanParams p = scan_params(h, a, h->partials, 1);
   const bool fused_tail = h->scan_mode == 0;
-  cudaError_t e;
-  {
-    fly::ScanParams tail = p;
-    tail.tickets = fused_tail ? h->tickets : nullptr;
-    int splits = 1;
-    if (h->cfg.logits_dtype == FLY_BF16)
-      e = launch_reduce<__nv_bfloat16>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
-                                       h->overlap != 0);
-    else
-      e = launch_reduce<float>(h, a->logits, stride, V, rows, h->forced_splits, h->partials, st, &splits, tail,
-                               h->overlap != 0);
-    if (e != cudaSuccess) return cuda_fail(h, e);
-    h->last_launches++;
-    h->last_splits = splits;
-    p.splits = splits;
-  }
+  p.tickets = fused_tail ? h->tickets : nullptr;
+  cudaError_t e = launch_reduce_any(h->cfg.logits_dtype, h->sm_count, a->logits, stride, V, rows, h->forced_splits,
+                                    kMaxSplits, h->partials, st, &p, p.scale, a->inputs_ready != 0);
+  if (e != cudaSuccess) return cuda_fail(h, e);
+  h->last_launches++;
   if (!fused_tail) {
     e = launch_scan(p, st);
     if (e != cudaSuccess) return cuda_fail(h, e);
@@ -598,8 +645,19 @@ fly_status_t fly_verify_run_host(fly_verify_t* h, const fly_verify_args_t* a, vo
     // packed into one block each way, so that a step costs one small copy in and one out
     const int64_t mb = h->cfg.max_batch, mk1 = h->cfg.max_k + 1;
     const size_t words = (size_t)(mb * (mk1 - 1) + 3 * mb + mb * mk1) + (size_t)(3 * mb + mb + mb + 4 * mb * mk1);
-    if ((e = cudaMalloc(&h->st_ints, words * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
-    if ((e = cudaMallocHost(&h->st_host, words * sizeof(int32_t))) != cudaSuccess) return cuda_fail(h, e);
+    int32_t* dev_block = nullptr;
+    int32_t* host_block = nullptr;
+    if ((e = cudaMalloc(&dev_block, words * sizeof(int32_t))) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return cuda_fail(h, e);
+    }
+    if ((e = cudaMallocHost(&host_block, words * sizeof(int32_t))) != cudaSuccess) {
+      (void)cudaGetLastError();
+      cudaFree(dev_block);
+      return cuda_fail(h, e);
+    }
+    h->st_ints = dev_block;  // both or neither
+    h->st_host = host_block;
   }
   const size_t hidden_bytes = a->logits ? 0 : (size_t)rows * h->cfg.hidden * 2;
   if (hidden_bytes > h->st_hidden_bytes) {
@@ -735,22 +793,17 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int64_t stride = a->row_stride ? a->row_stride : vocab;
-  const int64_t esz = logits_dtype == FLY_BF16 ? 2 : 4;
-  int splits = auto_splits(&h, rows, (int64_t)vocab * esz, kMaxSplits);
-  const int64_t room = FLY_STATIC_MAX_PIECES / rows;  // >= 1
-  if (splits > room) splits = (int)room;
+  const int64_t room = FLY_STATIC_MAX_PIECES / rows;  // Partial slots per row that fit, >= 1
+  const int cap = (int)(room < kMaxSplits ? room : kMaxSplits);
 
-  fly::ScanParams p = scan_params(&h, a, partials, splits);
+  fly::ScanParams p = scan_params(&h, a, partials, 1);
   p.tickets = tickets;
 
   // The arrival counters must start at zero, whatever an earlier call left behind.
-  cudaError_t e = cudaMemsetAsync(tickets, 0, FLY_STATIC_MAX_BATCH * 4, st);
+  cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)a->B * 4, st);
   if (e != cudaSuccess) return FLY_ERR_CUDA;
-  int used = 1;
-  if (logits_dtype == FLY_BF16)
-    e = launch_reduce<__nv_bfloat16>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
-  else
-    e = launch_reduce<float>(&h, a->logits, stride, vocab, rows, splits, partials, st, &used, p, false);
+  e = launch_reduce_any(logits_dtype, h.sm_count, a->logits, stride, vocab, rows, 0, cap, partials, st, &p, p.scale,
+                        a->inputs_ready != 0);
   return e == cudaSuccess ? FLY_OK : FLY_ERR_CUDA;
 }
 

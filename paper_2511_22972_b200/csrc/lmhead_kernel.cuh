@@ -97,6 +97,7 @@ struct Params {
   int num_kb;     // ceil(D / 64)
   int row0;       // first row of this launch in hidden / partials
   int w_kmajor;   // 0: weight is [D, V] (vocabulary contiguous, MN-major A); 1: weight is [V, D] (K-major A)
+  float scale;    // log2(e) / temperature: logit -> base-2 exponent
   Partial* partials;  // [rows, gridDim.x]: one partial state per position and CTA
   int* status;        // 0, or the code of the first wait that ran out
 };
@@ -192,7 +193,7 @@ struct Stream {
 };
 
 // Folds 16 consecutive vocabulary entries x[0..15] (the first one has index v0) into st.
-__device__ __forceinline__ void fold16(Stream& st, float (&x)[16], int v0) {
+__device__ __forceinline__ void fold16(Stream& st, float (&x)[16], int v0, float scale) {
   float lm = kMaskFloor;
 #pragma unroll
   for (int e = 0; e < 16; ++e) {
@@ -200,7 +201,7 @@ __device__ __forceinline__ void fold16(Stream& st, float (&x)[16], int v0) {
     lm = fmaxf(lm, x[e]);
   }
   if (lm > st.mx) {  // the maximum moves: rebase the sums and record the first entry that holds it
-    const float d = (st.mx - lm) * kLog2e;
+    const float d = (st.mx - lm) * scale;
     const float sc = ex2_approx(d);
     st.u = sc * fmaf(d, st.S, st.u);
     st.S *= sc;
@@ -211,11 +212,11 @@ __device__ __forceinline__ void fold16(Stream& st, float (&x)[16], int v0) {
       if (x[e] == lm) first = e;
     st.idx = v0 + first;
   }
-  const float nr = -st.mx * kLog2e;
+  const float nr = -st.mx * scale;
   float S0 = 0.f, S1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
   for (int e = 0; e < 16; e += 2) {
-    const float t0 = fmaf(x[e], kLog2e, nr), t1 = fmaf(x[e + 1], kLog2e, nr);
+    const float t0 = fmaf(x[e], scale, nr), t1 = fmaf(x[e + 1], scale, nr);
     const float e0 = ex2_approx(t0), e1 = ex2_approx(t1);
     S0 += e0;
     u0 = fmaf(e0, t0, u0);
@@ -412,7 +413,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
             for (int e = 0; e < 16; ++e)
               if (e >= limit) x[e] = kMaskFloor;
           }
-          fold16(st[k], x, v0);
+          fold16(st[k], x, v0, p.scale);
         }
       }
     }
@@ -430,7 +431,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     for (int pos = threadIdx.x; pos < p.R; pos += kEpiThreads) {
       Partial a = buf[pos * 8];
 #pragma unroll
-      for (int e = 1; e < 8; ++e) merge_partial(a, buf[pos * 8 + e]);
+      for (int e = 1; e < 8; ++e) merge_partial(a, buf[pos * 8 + e], p.scale);
       p.partials[(int64_t)(p.row0 + pos) * gridDim.x + blockIdx.x] = a;
     }
   }

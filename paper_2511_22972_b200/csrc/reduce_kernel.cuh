@@ -1,15 +1,38 @@
-// Row reduction of the FLy verification step: one streaming pass over a piece
-// of a logits row yields the running maximum, the softmax normaliser, the
-// weighted sum that gives the entropy (Eq. 5) and the greedy token (Eq. 1).
+// Row reduction of the FLy verification step: one streaming pass over the logits
+// yields, per row, the running maximum, the softmax normaliser, the weighted sum
+// that gives the entropy (Eq. 5) and the greedy token (Eq. 1).
 //
-// Work decomposition: unit = (row, split).  One thread block reduces one unit
-// and writes one 16-byte Partial.  Inside the block every warp streams its own
-// interleaved slices with 128-bit loads, UNROLL loads in flight per lane; the
-// warp keeps ONE reference exponent (its running maximum), so a slice costs one
-// warp-wide max (redux.sync) and the rescale / index search only runs when the
-// maximum actually moves (a handful of times per row).  Per element the steady
-// state is: widen, one FMA into the base-2 exponent, one MUFU ex2, two
-// accumulations.
+// Work decomposition ("flat partition").  The rows of one step are laid end to
+// end; a row holds `n` units (a unit is one 16-byte segment on the vector path,
+// one logit on the element-wise path).  The grid has G thread blocks, all
+// resident at once, and block b reduces the flat unit range [b*Q, (b+1)*Q): the
+// same number of bytes for every block, so that they finish together whatever
+// the number of rows is.  Where the range crosses a row boundary the block closes
+// the row's piece (one 16-byte Partial) and starts the next row.  In the flat
+// index space a row spans `span` >= n units (units past n do not exist): span = n
+// packs the rows densely (large steps: a block takes a long range, the odd row
+// boundary inside it costs little); span = s*Q cuts every row into exactly s
+// pieces that never cross a row (small steps, where a boundary inside a block
+// would lengthen its critical path by a whole slice).  Row r is covered by the
+// blocks (r*span)/Q .. ((r+1)*span-1)/Q, and piece k of a row is stored at
+// partials[row * slots + k].
+//
+// Memory pipeline (vector path).  Every warp owns a small ring in shared memory
+// that it fills with asynchronous 16-byte copies (cp.async): kDepth slices of
+// UNROLL*32 segments (2 KB each) are in flight per warp while it folds the oldest
+// one, 4 blocks x 8 warps per SM (128 KB in flight per SM, none of it in
+// registers).  A lane reads back exactly the bytes it copied, so the ring needs
+// no barrier.  The whole grid issues its first 2 x 2 KB per warp at once, and a
+// block that goes on into the next row starts that row's first slices before it
+// merges the finished piece: a grid that runs alone (one step of a decode loop)
+// has no second wave and no idle round trip at a row boundary.
+//
+// Arithmetic.  A warp keeps ONE reference exponent (its running maximum), so a
+// slice costs one warp-wide max (redux.sync) and the rescale / index search only
+// runs when the maximum actually moves (a handful of times per row).  Per pair of
+// logits the steady state is: widen (2), one packed FMA into the base-2
+// exponents, two MUFU ex2, one packed add and one packed FMA into the sums
+// (fma/add.f32x2: two fp32 operations per issue slot).
 #pragma once
 #include "fly_common.cuh"
 #include "scan_kernel.cuh"
@@ -18,41 +41,75 @@ namespace fly {
 
 constexpr int kReduceThreads = 256;
 constexpr int kReduceWarps = kReduceThreads / 32;
+constexpr int kReduceBlocksPerSM = 4;  // __launch_bounds__ below: <= 64 registers; measured against 3, 5 and 6
+constexpr int kDepth = 2;              // slices in flight per warp (3 and 4 measured: no faster)
+constexpr int kMaxPend = 8;            // finished pieces a block holds back before it writes them out
 
-// Per-warp streaming state.  S/u are per-lane (two accumulator pairs for ILP),
-// everything else is warp-uniform.
+// ---- packed fp32 pairs ------------------------------------------------------------------------
+using f2 = unsigned long long;  // two fp32 values in one 64-bit register: {lo, hi}
+
+__device__ __forceinline__ f2 pack2(float lo, float hi) {
+  f2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) {
+  f2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b) {
+  f2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ f2 mul2(f2 a, f2 b) {
+  f2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// Per-warp streaming state.  S2/u2 are per-lane pairs of accumulators, everything else is warp-uniform.
 struct WarpAcc {
   float cur_max;  // raw running maximum (warp-uniform)
-  float r;        // cur_max * log2(e): reference exponent of S and u
+  float r;        // cur_max * scale: reference exponent of S and u
+  float scale;    // log2(e) / temperature: logit -> base-2 exponent
   int best_idx;   // lowest index holding cur_max (warp-uniform)
-  float S0, u0, S1, u1;
+  f2 S2, u2;
 };
 
-__device__ __forceinline__ void acc_init(WarpAcc& a) {
+__device__ __forceinline__ void acc_init(WarpAcc& a, float scale) {
   a.cur_max = kMaskFloor;
-  a.r = kMaskFloor * kLog2e;
+  a.scale = scale;
+  a.r = kMaskFloor * scale;
   a.best_idx = kIdxNone;
-  a.S0 = a.u0 = a.S1 = a.u1 = 0.f;
+  a.S2 = pack2(0.f, 0.f);
+  a.u2 = pack2(0.f, 0.f);
 }
 
 // Moves the reference exponent to a larger maximum (warp-uniform call).
 __device__ __forceinline__ void acc_rebase(WarpAcc& a, float new_max) {
-  const float nr = new_max * kLog2e;
+  const float nr = new_max * a.scale;
   const float d = a.r - nr;  // < 0, finite
   const float sc = ex2_approx(d);
-  a.u0 = sc * fmaf(d, a.S0, a.u0);
-  a.u1 = sc * fmaf(d, a.S1, a.u1);
-  a.S0 *= sc;
-  a.S1 *= sc;
+  const f2 d2 = pack2(d, d), sc2 = pack2(sc, sc);
+  a.u2 = mul2(sc2, fma2(d2, a.S2, a.u2));
+  a.S2 = mul2(a.S2, sc2);
   a.r = nr;
   a.cur_max = new_max;
 }
 
-__device__ __forceinline__ void acc_add(float x, float nr, float& S, float& u) {
-  const float t = fmaf(x, kLog2e, nr);  // nr = -r
-  const float e = ex2_approx(t);
-  S += e;
-  u = fmaf(e, t, u);
+// Adds the pair of logits (x0, x1): t = x * scale - r, S += 2^t, u += 2^t * t.
+__device__ __forceinline__ void acc_add2(WarpAcc& a, float x0, float x1, f2 sc2, f2 nr2) {
+  const f2 t2 = fma2(pack2(x0, x1), sc2, nr2);
+  float t0, t1;
+  unpack2(t2, t0, t1);
+  const f2 e2 = pack2(ex2_approx(t0), ex2_approx(t1));
+  a.S2 = add2(a.S2, e2);
+  a.u2 = fma2(e2, t2, a.u2);
 }
 
 // ---------------------------------------------------------------------------
@@ -63,14 +120,6 @@ __device__ __forceinline__ void acc_add(float x, float nr, float& S, float& u) {
 template <typename T> struct Seg;
 template <> struct Seg<__nv_bfloat16> { static constexpr int kElems = 8; };
 template <> struct Seg<float> { static constexpr int kElems = 4; };
-
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
-  uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.L2::128B.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-               : "l"(p));
-  return v;
-}
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -88,12 +137,29 @@ __device__ __forceinline__ uint32_t bf2_max_nan(uint32_t a, uint32_t b) {
 
 constexpr uint32_t kNegInf2 = 0xff80ff80u;  // bf16 (-inf, -inf)
 
-// Folds one warp slice of UNROLL*32 segments of bf16 logits, already in registers, into the
-// warp's running state.  w[j] is segment seg0 + j*32 + lane of the row (8 logits).
+__device__ __forceinline__ uint32_t smem_addr_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Asynchronous 16-byte copy global -> shared (bypasses L1, no register staging).
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
+  asm volatile("cp.async.cg.shared.global.L2::128B [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// First half of folding a slice of bf16 logits (w[j] = segment seg0 + j*32 + lane of the row, 8 logits;
+// segments at or past seg_end do not belong to the piece): masks and clamps the data and returns the
+// lane's maximum.  Masked entries are clamped to the floor (NaN survives the clamp and ends in S).
 template <int UNROLL>
-__device__ __forceinline__ void fold_slice_bf16(WarpAcc& a, uint32_t (&w)[UNROLL][4], int seg0, int lane) {
-  constexpr uint32_t kFloor2 = 0xc974c974u;   // bf16(kMaskFloor) twice
-  // clamp masked entries to the floor (NaN survives the clamp and ends in S)
+__device__ __forceinline__ float slice_max_bf16(uint32_t (&w)[UNROLL][4], int seg0, int seg_end, int lane) {
+  constexpr uint32_t kFloor2 = 0xc974c974u;  // bf16(kMaskFloor) twice
+  if (seg0 + UNROLL * 32 > seg_end) {        // ragged slice (warp-uniform)
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j)
+      if (seg0 + j * 32 + lane >= seg_end) w[j][0] = w[j][1] = w[j][2] = w[j][3] = kNegInf2;
+  }
   uint32_t lm2 = kFloor2;
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j)
@@ -102,7 +168,12 @@ __device__ __forceinline__ void fold_slice_bf16(WarpAcc& a, uint32_t (&w)[UNROLL
       w[j][c] = bf2_max_nan(w[j][c], kFloor2);
       lm2 = bf2_max(lm2, w[j][c]);
     }
-  const float lm = fmaxf(bf16lo(lm2), bf16hi(lm2));
+  return fmaxf(bf16lo(lm2), bf16hi(lm2));
+}
+
+// Second half: warp maximum, rebase when it moved, then the exponentials.
+template <int UNROLL>
+__device__ __forceinline__ void slice_sum_bf16(WarpAcc& a, const uint32_t (&w)[UNROLL][4], float lm, int seg0, int lane) {
   const float wm = warp_max_f32(lm);
   if (wm > a.cur_max) {  // warp-uniform, rare after the first slices
     acc_rebase(a, wm);
@@ -119,28 +190,34 @@ __device__ __forceinline__ void fold_slice_bf16(WarpAcc& a, uint32_t (&w)[UNROLL
     }
     a.best_idx = (int)warp_min_u32(first);
   }
-  const float nr = -a.r;
+  const f2 nr2 = pack2(-a.r, -a.r), sc2 = pack2(a.scale, a.scale);
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      acc_add(bf16lo(w[j][c]), nr, a.S0, a.u0);
-      acc_add(bf16hi(w[j][c]), nr, a.S1, a.u1);
-    }
+    for (int c = 0; c < 4; ++c) acc_add2(a, bf16lo(w[j][c]), bf16hi(w[j][c]), sc2, nr2);
 }
 
-
-// The same for fp32 logits: x[j] is segment seg0 + j*32 + lane of the row (4 logits).
+// The same two halves for fp32 logits: w[j] holds 4 logits as raw bits.
 template <int UNROLL>
-__device__ __forceinline__ void fold_slice_f32(WarpAcc& a, float (&x)[UNROLL][4], int seg0, int lane) {
+__device__ __forceinline__ float slice_max_f32(uint32_t (&w)[UNROLL][4], int seg0, int seg_end, int lane) {
+  if (seg0 + UNROLL * 32 > seg_end) {
+#pragma unroll
+    for (int j = 0; j < UNROLL; ++j)
+      if (seg0 + j * 32 + lane >= seg_end) w[j][0] = w[j][1] = w[j][2] = w[j][3] = 0xff800000u;
+  }
   float lm = kMaskFloor;
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j)
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-      x[j][c] = max_nan_f32(x[j][c], kMaskFloor);
-      lm = fmaxf(lm, x[j][c]);
+      const float x = max_nan_f32(__uint_as_float(w[j][c]), kMaskFloor);
+      w[j][c] = __float_as_uint(x);
+      lm = fmaxf(lm, x);
     }
+  return lm;
+}
+template <int UNROLL>
+__device__ __forceinline__ void slice_sum_f32(WarpAcc& a, const uint32_t (&w)[UNROLL][4], float lm, int seg0, int lane) {
   const float wm = warp_max_f32(lm);
   if (wm > a.cur_max) {
     acc_rebase(a, wm);
@@ -150,54 +227,15 @@ __device__ __forceinline__ void fold_slice_f32(WarpAcc& a, float (&x)[UNROLL][4]
       for (int j = UNROLL - 1; j >= 0; --j)
 #pragma unroll
         for (int c = 3; c >= 0; --c)
-          if (x[j][c] == wm) first = (uint32_t)(seg0 + j * 32 + lane) * 4u + (uint32_t)c;
+          if (__uint_as_float(w[j][c]) == wm) first = (uint32_t)(seg0 + j * 32 + lane) * 4u + (uint32_t)c;
     }
     a.best_idx = (int)warp_min_u32(first);
   }
-  const float nr = -a.r;
+  const f2 nr2 = pack2(-a.r, -a.r), sc2 = pack2(a.scale, a.scale);
 #pragma unroll
   for (int j = 0; j < UNROLL; ++j) {
-    acc_add(x[j][0], nr, a.S0, a.u0);
-    acc_add(x[j][1], nr, a.S1, a.u1);
-    acc_add(x[j][2], nr, a.S0, a.u0);
-    acc_add(x[j][3], nr, a.S1, a.u1);
-  }
-}
-
-
-// Loads UNROLL segments, 32 segments apart, starting at p (a lane's pointer into a full slice).
-template <int UNROLL>
-__device__ __forceinline__ void load_full_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ p) {
-#pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    const uint4 q = ld_stream(p + j * 32);  // constant offsets: one pointer per slice
-    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-  }
-}
-// The same for a slice that runs past seg_end: segments at or past seg_end read as -inf.
-template <int UNROLL>
-__device__ __forceinline__ void load_ragged_slice(uint32_t (&w)[UNROLL][4], const uint4* __restrict__ row, int seg0,
-                                                  int seg_end, int lane, uint32_t fill) {
-#pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    const int s = seg0 + j * 32 + lane;
-    uint4 q = make_uint4(fill, fill, fill, fill);
-    if (s < seg_end) q = ld_stream(row + s);
-    w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
-  }
-}
-
-template <typename T, int UNROLL>
-__device__ __forceinline__ void fold_slice(WarpAcc& a, uint32_t (&w)[UNROLL][4], int seg0, int lane) {
-  if constexpr (sizeof(T) == 2) {
-    fold_slice_bf16<UNROLL>(a, w, seg0, lane);
-  } else {
-    float x[UNROLL][4];
-#pragma unroll
-    for (int j = 0; j < UNROLL; ++j)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) x[j][c] = __uint_as_float(w[j][c]);
-    fold_slice_f32<UNROLL>(a, x, seg0, lane);
+    acc_add2(a, __uint_as_float(w[j][0]), __uint_as_float(w[j][1]), sc2, nr2);
+    acc_add2(a, __uint_as_float(w[j][2]), __uint_as_float(w[j][3]), sc2, nr2);
   }
 }
 
@@ -228,19 +266,48 @@ __device__ __forceinline__ void warp_slice_scalar(WarpAcc& a, const T* __restric
     }
     a.best_idx = (int)warp_min_u32(first);
   }
-  const float nr = -a.r;
+  const f2 nr2 = pack2(-a.r, -a.r), sc2 = pack2(a.scale, a.scale);
+  // out-of-range lanes hold the floor: 2^(floor*scale - r) = 0 unless the whole
+  // piece is masked, in which case the piece vanishes when merged
+  if constexpr (UNROLL == 1) {
+    acc_add2(a, x[0], kMaskFloor, sc2, nr2);
+  } else {
 #pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    // out-of-range lanes hold the floor: 2^(floor*log2e - r) = 0 unless the whole
-    // piece is masked, in which case the piece vanishes when merged
-    acc_add(x[j], nr, a.S0, a.u0);
+    for (int j = 0; j < UNROLL; j += 2) acc_add2(a, x[j], x[j + 1], sc2, nr2);
   }
 }
 
-// Lanes -> warp -> block, then one Partial per unit.
-__device__ __forceinline__ void block_finish(const WarpAcc& a, Partial* __restrict__ out, int lane, int warp) {
-  __shared__ Partial sm[kReduceWarps];
-  float S = a.S0 + a.S1, u = a.u0 + a.u1;
+// One piece on the element-wise path: logits [e_begin, e_end) of the row.
+template <typename T, int UNROLL>
+__device__ __forceinline__ void reduce_piece_scalar(WarpAcc& a, const T* __restrict__ rp, int e_begin, int e_end, int lane,
+                                                    int warp) {
+  constexpr int kSlice = UNROLL * 32;
+  for (int e0 = e_begin + warp * kSlice; e0 < e_end; e0 += kReduceWarps * kSlice)
+    warp_slice_scalar<T, UNROLL>(a, rp, e0, e_end, lane);
+}
+
+// Geometry of one launch (see the head of this file).
+struct ReducePlan {
+  int64_t n;       // units per row
+  int64_t span;    // units a row takes in the flat index space (>= n)
+  int64_t Q;       // units per block
+  int64_t total;   // rows * span
+  int slots;       // Partial slots per row (>= the largest number of pieces of any row)
+  int V;
+  int64_t row_stride;  // elements
+  float scale;     // log2(e) / temperature
+  int wait_first;  // 1: wait for the previous kernel in the stream before the first read (plain stream
+                   //    order); 0: the logits are known to be complete, wait only before the first write
+};
+
+// Lanes -> warp -> block; warp 0 / lane 0 ends up with the piece's Partial.  sm: kReduceWarps Partials of
+// shared memory; consecutive pieces of a block alternate between two such buffers, so one barrier per
+// piece is enough.
+__device__ __forceinline__ Partial block_finish(const WarpAcc& a, Partial* sm, int lane, int warp) {
+  float S0, S1, u0, u1;
+  unpack2(a.S2, S0, S1);
+  unpack2(a.u2, u0, u1);
+  float S = S0 + S1, u = u0 + u1;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     S += __shfl_xor_sync(0xffffffffu, S, o);
@@ -252,29 +319,37 @@ __device__ __forceinline__ void block_finish(const WarpAcc& a, Partial* __restri
     sm[warp] = p;
   }
   __syncthreads();
+  Partial p = empty_partial();
   if (warp == 0) {
-    Partial p = lane < kReduceWarps ? sm[lane] : empty_partial();
+    if (lane < kReduceWarps) p = sm[lane];
 #pragma unroll
     for (int o = kReduceWarps / 2; o > 0; o >>= 1) {
       Partial q = shfl_xor_partial(p, o);
-      merge_partial(p, q);
+      merge_partial(p, q, a.scale);
     }
-    if (lane == 0) *out = p;
   }
+  return p;
 }
 
-// Fused tail: the block that completes a sequence's last unit verifies the
-// sequence.  Called by every thread after block_finish; only warp 0 acts.
-__device__ __forceinline__ void sequence_tail(const ScanParams& p, int row, int lane, int warp) {
-  __shared__ int sm_y[kMaxRows];
-  if (warp != 0 || p.tickets == nullptr) return;
+// A finished piece that has not been written out yet.
+struct __align__(16) Pending {
+  Partial p;
+  int row, slot;
+  unsigned units;
+  int pad;
+};
+
+// Fused tail: the block that completes a sequence verifies it.  A sequence's arrival counter counts the
+// units (segments or logits) of its K+1 rows that have been reduced; the block whose piece brings it to
+// (K+1) * n has seen every other piece's ticket, hence (after the fences) every other Partial.  Called by
+// warp 0 once the piece's Partial is in global memory.
+__device__ __forceinline__ void sequence_tail(const ScanParams& p, int row, unsigned units, int lane, int* sm_y) {
   const int K1 = p.K + 1;
   const int b = row / K1;
   unsigned last = 0;
   if (lane == 0) {
-    __threadfence();  // the partial written above is visible before the ticket is taken
-    const unsigned t = atomicAdd(p.tickets + b, 1u);
-    last = (t == (unsigned)(K1 * p.splits) - 1u);
+    const unsigned t = atomicAdd(p.tickets + b, units);
+    last = (t + units == (unsigned)K1 * (unsigned)p.units_per_row);
     if (last) {
       p.tickets[b] = 0;  // ready for the next launch
       __threadfence();
@@ -287,76 +362,160 @@ __device__ __forceinline__ void sequence_tail(const ScanParams& p, int row, int 
   }
 }
 
-// grid.x = rows * splits.  Vector path.
-//   segs_per_split  whole segments per unit (the last unit of a row may be short)
-//   nseg            whole segments in a row; elements [nseg*kElems, V) are the ragged tail
-template <typename T, int UNROLL>
-__global__ void __launch_bounds__(kReduceThreads)
-reduce_rows_vec(const T* __restrict__ logits, int64_t row_stride, int V, int nseg, int splits, int segs_per_split,
-                Partial* __restrict__ partials, const __grid_constant__ ScanParams tail) {
-  constexpr int kE = Seg<T>::kElems;
-  const int unit = blockIdx.x;
-  const int row = unit / splits, split = unit - row * splits;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const T* rp = logits + (int64_t)row * row_stride;
-  const uint4* rv = reinterpret_cast<const uint4*>(rp);
-  const int seg_begin = split * segs_per_split;
-  const int seg_end = min(nseg, seg_begin + segs_per_split);
-
-  // Let a programmatic dependent (the stand-alone scan kernel, or the next
-  // step's reduction) get scheduled; it waits for this grid's completion before
-  // it touches anything this grid writes.
-  asm volatile("griddepcontrol.launch_dependents;");
-
-  WarpAcc a;
-  acc_init(a);
-  constexpr int kSlice = UNROLL * 32;
-  constexpr uint32_t kFill = sizeof(T) == 2 ? kNegInf2 : 0xff800000u;
-  constexpr int kStride = kReduceWarps * kSlice;
-  int s0 = seg_begin + warp * kSlice;
-  const uint4* ptr = rv + s0 + lane;
-  for (; s0 + kSlice <= seg_end; s0 += kStride, ptr += kStride) {  // full slices: no predicates
-    uint32_t w[UNROLL][4];
-    load_full_slice<UNROLL>(w, ptr);
-    fold_slice<T, UNROLL>(a, w, s0, lane);
-  }
-  if (s0 < seg_end) {  // at most one slice of a warp runs past the end of the piece
-    uint32_t w[UNROLL][4];
-    load_ragged_slice<UNROLL>(w, rv, s0, seg_end, lane, kFill);
-    fold_slice<T, UNROLL>(a, w, s0, lane);
-  }
-  // ragged tail (fewer than kElems logits): last unit of the row, last warp
-  if (split == splits - 1 && warp == kReduceWarps - 1 && nseg * kE < V)
-    warp_slice_scalar<T, 1>(a, rp, nseg * kE, V, lane);
-  // Everything above only reads the logits.  When this grid was launched as a
-  // programmatic dependent of the previous kernel in the stream, wait for that
-  // kernel to complete before the first write (scratch and outputs are shared
-  // between consecutive steps).  Otherwise this returns at once.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  block_finish(a, partials + unit, lane, warp);
-  sequence_tail(tail, row, lane, warp);
+// Writes the held-back pieces out and takes their tickets (warp 0).
+__device__ __forceinline__ void flush_pending(const Pending* pend, int np, int slots, Partial* __restrict__ partials,
+                                              const ScanParams& tail, int lane, int* sm_y) {
+  if (lane < np) partials[(int64_t)pend[lane].row * slots + pend[lane].slot] = pend[lane].p;
+  if (tail.tickets == nullptr) return;
+  __threadfence();  // the partials written above are visible ...
+  __syncwarp();
+  __threadfence();  // ... before lane 0 takes any ticket
+  for (int k = 0; k < np; ++k) sequence_tail(tail, pend[k].row, pend[k].units, lane, sm_y);
 }
 
-// grid.x = rows * splits.  Any alignment, any V.
-template <typename T, int UNROLL>
-__global__ void __launch_bounds__(kReduceThreads)
-reduce_rows_scalar(const T* __restrict__ logits, int64_t row_stride, int V, int splits, int elems_per_split,
-                   Partial* __restrict__ partials, const __grid_constant__ ScanParams tail) {
-  const int unit = blockIdx.x;
-  const int row = unit / splits, split = unit - row * splits;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const T* rp = logits + (int64_t)row * row_stride;
-  const int e_begin = split * elems_per_split;
-  const int e_end = min(V, e_begin + elems_per_split);
-  asm volatile("griddepcontrol.launch_dependents;");
-  WarpAcc a;
-  acc_init(a);
+// grid.x = ceil(total / Q).  VEC: rows are 16-byte structured (a unit is a segment); else any alignment, any V.
+template <typename T, int UNROLL, bool VEC>
+__global__ void __launch_bounds__(kReduceThreads, kReduceBlocksPerSM)
+reduce_rows_flat(const T* __restrict__ logits, const __grid_constant__ ReducePlan g, Partial* __restrict__ partials,
+                 const __grid_constant__ ScanParams tail) {
+  constexpr int kE = Seg<T>::kElems;
   constexpr int kSlice = UNROLL * 32;
-  for (int e0 = e_begin + warp * kSlice; e0 < e_end; e0 += kReduceWarps * kSlice)
-    warp_slice_scalar<T, UNROLL>(a, rp, e0, e_end, lane);
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  block_finish(a, partials + unit, lane, warp);
-  sequence_tail(tail, row, lane, warp);
+  constexpr int kStride = kReduceWarps * kSlice;
+  extern __shared__ __align__(16) uint4 ring[];  // VEC: kReduceWarps * kDepth * kSlice segments
+  __shared__ Partial sm_part[2][kReduceWarps];
+  __shared__ Pending pend[kMaxPend];
+  __shared__ int sm_y[kMaxRows];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  // The grid is launched as a programmatic dependent of the previous kernel in the stream.  Plain
+  // stream order: wait for that kernel to complete (and its writes to be visible) before anything is
+  // read.  With inputs_ready the reads start at once and the wait comes before the first write.
+  bool waited = g.wait_first != 0;
+  if (waited) asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Let the next kernel in the stream get scheduled early if it asks for that; it waits for this
+  // grid's completion before it touches anything this grid writes.
+  asm volatile("griddepcontrol.launch_dependents;");
+
+  const int64_t f0 = (int64_t)blockIdx.x * g.Q;
+  const int64_t f_end = min(f0 + g.Q, g.total);
+  int row = (int)(f0 / g.span);
+  int u0 = (int)(f0 - (int64_t)row * g.span);                              // first unit of this block's piece inside the row
+  int slot = (int)((int64_t)blockIdx.x - ((int64_t)row * g.span) / g.Q);   // pieces of the row that earlier blocks hold
+  int u1 = (int)min(g.n, (int64_t)u0 + (f_end - f0));                      // end of the piece inside the row
+  // flat units of this block not yet assigned to a piece (a row ends at its span, not at n)
+  int64_t left = f_end - f0;
+  int64_t take = min((int64_t)g.span - u0, left);                          // flat units the current piece takes
+
+  // Copy side of the pipeline.  A warp's slices of the piece [pu0, pu1) of the row at `prow` start at
+  // ps = pu0 + warp * kSlice and lie kStride apart; issue() copies the next one into a ring stage.
+  const uint32_t ring_warp = smem_addr_u32(ring) + (uint32_t)((warp * kDepth * kSlice + lane) * 16);
+  const uint4* psrc = nullptr;
+  int ps = 0, pend_seg = 0;
+  auto open_piece = [&](int prow, int pu0, int pu1) {
+    psrc = reinterpret_cast<const uint4*>(logits + (int64_t)prow * g.row_stride) + lane;
+    ps = pu0 + warp * kSlice;
+    pend_seg = pu1;
+  };
+  auto issue = [&](int stage) {
+    if (ps < pend_seg) {
+      const uint32_t dst = ring_warp + (uint32_t)(stage * kSlice * 16);
+      if (ps + kSlice <= pend_seg) {
+#pragma unroll
+        for (int j = 0; j < UNROLL; ++j) cp_async16(dst + j * 512, psrc + ps + j * 32);
+      } else {
+#pragma unroll
+        for (int j = 0; j < UNROLL; ++j)
+          if (ps + j * 32 + lane < pend_seg) cp_async16(dst + j * 512, psrc + ps + j * 32);
+      }
+      ps += kStride;
+    }
+    cp_async_commit();  // one group per call, empty or not: the folding side counts groups
+  };
+  if constexpr (VEC) {
+    open_piece(row, u0, u1);
+#pragma unroll
+    for (int d = 0; d < kDepth; ++d) issue(d);
+  }
+
+  // The acceptance scan at the end of the step reads draft tokens and carried state, which nothing has
+  // touched yet: pull them into L2 now so that the last block does not wait on DRAM for them.
+  if (tail.tickets != nullptr && (int)blockIdx.x < tail.B && warp == 1) {
+    const int32_t* d = tail.draft + (int64_t)blockIdx.x * tail.K;
+    if (lane * 32 < tail.K) asm volatile("prefetch.global.L2 [%0];" ::"l"(d + lane * 32));
+    if (lane == 31 && tail.state_in) asm volatile("prefetch.global.L2 [%0];" ::"l"(tail.state_in + (int64_t)blockIdx.x * 3));
+  }
+
+  int parity = 0, np = 0;
+  while (true) {
+    const T* rp = logits + (int64_t)row * g.row_stride;
+    WarpAcc a;
+    acc_init(a, g.scale);
+    left -= take;
+    if constexpr (VEC) {
+      int stage = 0;
+      for (int s0 = u0 + warp * kSlice; s0 < u1; s0 += kStride) {
+        cp_async_wait<kDepth - 1>();  // the oldest slice in flight has landed
+        uint32_t w[UNROLL][4];
+        const uint4* src = ring + (warp * kDepth + stage) * kSlice + lane;
+#pragma unroll
+        for (int j = 0; j < UNROLL; ++j) {
+          const uint4 q = src[j * 32];
+          w[j][0] = q.x; w[j][1] = q.y; w[j][2] = q.z; w[j][3] = q.w;
+        }
+        float lm;
+        if constexpr (sizeof(T) == 2) lm = slice_max_bf16<UNROLL>(w, s0, u1, lane);
+        else lm = slice_max_f32<UNROLL>(w, s0, u1, lane);
+        // every register of the slice has been consumed once, so the stage's bytes are out of shared
+        // memory: refill it with the slice kDepth ahead
+        issue(stage);
+        if constexpr (sizeof(T) == 2) slice_sum_bf16<UNROLL>(a, w, lm, s0, lane);
+        else slice_sum_f32<UNROLL>(a, w, lm, s0, lane);
+        stage = stage + 1 == kDepth ? 0 : stage + 1;
+      }
+      // This warp's ring is empty now.  If the block goes on into the next row, start that piece's first
+      // slices before the block-wide merge below, so that the row boundary costs no memory round trip.
+      if (left > 0) {
+        cp_async_wait<0>();
+        open_piece(row + 1, 0, (int)min(g.n, left));
+#pragma unroll
+        for (int d = 0; d < kDepth; ++d) issue(d);
+      }
+      // ragged tail (fewer than kElems logits): the piece that ends the row, last warp
+      if (u1 == (int)g.n && warp == kReduceWarps - 1 && (int)g.n * kE < g.V) warp_slice_scalar<T, 1>(a, rp, (int)g.n * kE, g.V, lane);
+    } else {
+      reduce_piece_scalar<T, UNROLL>(a, rp, u0, u1, lane, warp);
+    }
+    const Partial p = block_finish(a, sm_part[parity], lane, warp);
+    if (warp == 0 && lane == 0) {
+      Pending q;
+      q.p = p; q.row = row; q.slot = slot; q.units = (unsigned)(u1 - u0); q.pad = 0;
+      pend[np] = q;
+    }
+    ++np;
+    parity ^= 1;
+    const bool done = left <= 0;
+    if (np == kMaxPend || done) {
+      // Everything so far only read the logits.  Scratch and outputs are shared with the previous step:
+      // with inputs_ready its kernel may still be running, so wait for it before the first write.
+      if (!waited) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        waited = true;
+      }
+      if (warp == 0) {
+        __syncwarp();
+        flush_pending(pend, np, g.slots, partials, tail, lane, sm_y);
+        __syncwarp();
+      }
+      np = 0;
+    }
+    if (done) break;
+    ++row;
+    u0 = 0;
+    u1 = (int)min(g.n, left);
+    take = min((int64_t)g.span, left);
+    slot = 0;
+  }
+  if constexpr (VEC) cp_async_wait<0>();
 }
 
 }  // namespace fly

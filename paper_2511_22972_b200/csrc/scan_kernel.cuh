@@ -20,7 +20,14 @@ constexpr int kMaxRows = 64;  // K + 1 <= 64
 
 struct ScanParams {
   int B, K, V;
-  int splits;
+  int splits;               // Partial slots per row
+  // Flat partition of the row reduction (Q > 0): a row holds units_per_row units and spans row_span >= units_per_row
+  // positions of the flat index space; thread block b reduced the flat range [b*Q, (b+1)*Q), so row r has
+  // ((r+1)*span - 1)/Q - (r*span)/Q + 1 pieces in its first slots.  Q == 0: every row has exactly `splits` pieces.
+  int64_t units_per_row;
+  int64_t row_span;
+  int64_t Q;
+  float scale;              // log2(e) / temperature (exponent unit of the partial states)
   const Partial* partials;  // [B*(K+1), splits]
   unsigned int* tickets;    // [B] arrival counters for the fused tail (zero between launches), or null
   const int32_t* draft;     // [B, K]
@@ -86,6 +93,13 @@ __device__ __forceinline__ Partial ld_partial_cg(const Partial* p) {
   return q;
 }
 
+// Number of pieces the flat partition cut row `row` into (see ScanParams).
+__device__ __forceinline__ int pieces_of_row(int64_t row, int64_t span, int64_t Q, int fixed) {
+  if (Q <= 0) return fixed;
+  const int64_t f0 = row * span;
+  return (int)((f0 + span - 1) / Q - f0 / Q) + 1;
+}
+
 // One warp verifies sequence b.  sm_y: kMaxRows ints of shared memory private to the warp.
 __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, int lane, int* sm_y) {
   const int K = p.K, K1 = p.K + 1;
@@ -111,13 +125,14 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
     if (i < K1) {
       const int64_t row = (int64_t)b * K1 + i;
       const Partial* pp = p.partials + row * p.splits;
+      const int pieces = pieces_of_row(row, p.row_span, p.Q, p.splits);
       Partial acc = empty_partial();
-      for (int s0 = 0; s0 < p.splits; s0 += 4) {  // four independent loads in flight
+      for (int s0 = 0; s0 < pieces; s0 += 4) {  // four independent loads in flight
         Partial q[4];
 #pragma unroll
-        for (int t = 0; t < 4; ++t) q[t] = (s0 + t < p.splits) ? ld_partial_cg(pp + s0 + t) : empty_partial();
+        for (int t = 0; t < 4; ++t) q[t] = (s0 + t < pieces) ? ld_partial_cg(pp + s0 + t) : empty_partial();
 #pragma unroll
-        for (int t = 0; t < 4; ++t) merge_partial(acc, q[t]);
+        for (int t = 0; t < 4; ++t) merge_partial(acc, q[t], p.scale);
       }
       // entropy is non-negative; rounding may leave -1e-7 on a one-hot row
       const float H = fmaxf(kLn2 * (log2f(acc.S) - acc.u / acc.S), 0.f);
@@ -177,16 +192,18 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
 // is in[r * row_stride + j * part_stride].  The fused LM-head kernel leaves one partial state per row
 // and CTA, a vocabulary-parallel target one per row and rank; folding them with 32 lanes in parallel
 // keeps the acceptance scan's per-lane loop short.  idx_offset is added to the winning index (a
-// vocabulary shard reports global token ids).
+// vocabulary shard reports global token ids).  With Q > 0 the number of parts of a row follows from
+// the flat partition of the row reduction (see ScanParams) instead of being n_fixed.
 constexpr int kFoldThreads = 128;
-__global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __restrict__ in, int n, int64_t row_stride,
+__global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __restrict__ in, int n_fixed, int64_t row_stride,
                                                               int64_t part_stride, Partial* __restrict__ out, int rows,
-                                                              int idx_offset) {
+                                                              int idx_offset, float scale, int64_t row_span, int64_t Q) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (kFoldThreads / 32) + (threadIdx.x >> 5);
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the producer grid has completed
   asm volatile("griddepcontrol.launch_dependents;");
   if (row >= rows) return;
+  const int n = pieces_of_row(row, row_span, Q, n_fixed);
   const Partial* src = in + (int64_t)row * row_stride;
   Partial acc = empty_partial();
   for (int j0 = 0; j0 < n; j0 += 128) {  // four independent loads in flight per lane
@@ -195,12 +212,12 @@ __global__ void __launch_bounds__(kFoldThreads) fold_partials(const Partial* __r
     for (int t = 0; t < 4; ++t)
       q[t] = (j0 + t * 32 + lane < n) ? ld_partial_cg(src + (int64_t)(j0 + t * 32 + lane) * part_stride) : empty_partial();
 #pragma unroll
-    for (int t = 0; t < 4; ++t) merge_partial(acc, q[t]);
+    for (int t = 0; t < 4; ++t) merge_partial(acc, q[t], scale);
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const Partial q = shfl_xor_partial(acc, o);
-    merge_partial(acc, q);
+    merge_partial(acc, q, scale);
   }
   if (lane == 0) {
     if (acc.idx != kIdxNone) acc.idx += idx_offset;

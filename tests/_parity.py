@@ -23,22 +23,24 @@ def draw(w, step=0, setting=0, device="cuda", thetas=None, guard=True):
     return logits, draft
 
 
-def gpu_step(fv, logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats", host=False):
+def gpu_step(fv, logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats", host=False,
+             temperature=0.0, inputs_ready=False):
     B, K1, V = logits.shape
     out = VerifyBuffers(B, K1 - 1, logits.device if not host else "cpu", pinned=host)
     if state is not None:
         out.state.copy_(torch.as_tensor(state, dtype=torch.int32))
     verify(fv, logits, draft, out, theta=theta, W=W, theta_unit=theta_unit, boundary=boundary,
-           stream=torch.cuda.current_stream().cuda_stream, host=host)
+           stream=torch.cuda.current_stream().cuda_stream, host=host, temperature=temperature,
+           inputs_ready=inputs_ready)
     torch.cuda.synchronize()
     return out
 
 
-def oracle_step(logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats"):
+def oracle_step(logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats", temperature=1.0):
     B, K1, V = logits.shape
     x = logits.double().cpu().numpy()
     return O.verify_batch(x, draft.cpu().numpy(), theta, W, theta_unit=theta_unit, boundary=boundary,
-                          state_in=None if state is None else np.asarray(state))
+                          state_in=None if state is None else np.asarray(state), temperature=temperature)
 
 
 def assert_parity(out, ref, what=""):
@@ -60,7 +62,9 @@ def assert_parity(out, ref, what=""):
     return float(err.max()) if err.size else 0.0
 
 
-def check(fv, logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats", what="", host=False):
-    out = gpu_step(fv, logits, draft, theta, W, boundary, state, theta_unit, host=host)
-    ref = oracle_step(logits, draft, theta, W, boundary, state, theta_unit)
+def check(fv, logits, draft, theta, W, boundary="reject", state=None, theta_unit="nats", what="", host=False,
+          temperature=0.0, inputs_ready=False):
+    out = gpu_step(fv, logits, draft, theta, W, boundary, state, theta_unit, host=host, temperature=temperature,
+                   inputs_ready=inputs_ready)
+    ref = oracle_step(logits, draft, theta, W, boundary, state, theta_unit, temperature=temperature or 1.0)
     return assert_parity(out, ref, what), out, ref

@@ -1,6 +1,7 @@
-"""The benchmark workloads at their FULL sizes, in the launch configuration bench.py times (consecutive
-steps overlapped, outputs of a step read back after later steps were enqueued), compared with the fp64
-oracle element by element.  The fused LM-head workload is in test_gpu_fused.py."""
+"""The benchmark workloads at their FULL sizes, in both launch configurations bench.py times (plain stream
+order, and consecutive steps overlapped over resident inputs; outputs of a step are read back after later steps
+were enqueued), compared with the fp64 oracle element by element.  The fused LM-head workload is in
+test_gpu_fused.py."""
 import numpy as np
 import pytest
 import torch
@@ -13,10 +14,11 @@ DEV = "cuda"
 
 
 def run_overlapped(fv, steps, theta, W, boundary="reject", chain=False):
-    """Enqueues all steps back to back on one stream, then compares every step with the oracle.
+    """Enqueues all steps back to back on one stream, then compares every step with the oracle; the even steps
+    in plain stream order, the odd ones with inputs_ready (they may read while the step before them drains).
     chain=True: one state buffer is carried from step to step (carry mode)."""
     st = torch.cuda.current_stream().cuda_stream
-    fv.set_stream_overlap(True)
+    torch.cuda.synchronize()                         # every step's inputs are complete before the first launch
     B, K1, _ = steps[0][0].shape
     outs = [VerifyBuffers(B, K1 - 1, DEV) for _ in steps]
     state = outs[0].state
@@ -24,7 +26,8 @@ def run_overlapped(fv, steps, theta, W, boundary="reject", chain=False):
     for (logits, draft), out in zip(steps, outs):
         if chain:
             out.state = state                        # every step reads and writes the same carried state
-        verify(fv, logits, draft, out, theta=theta, W=W, boundary=boundary, stream=st)
+        verify(fv, logits, draft, out, theta=theta, W=W, boundary=boundary, stream=st,
+               inputs_ready=len(snapshots) % 2 == 1 if chain else (outs.index(out) % 2 == 1))
         if chain:
             snapshots.append(state.clone())          # stream-ordered copy of the state after this step
     torch.cuda.synchronize()
@@ -94,12 +97,12 @@ def test_repeated_steps_are_bit_identical():
 
     w = S.LLAMA3
     fv = FlyVerify(w.B, w.K, w.V, w.dtype)
-    fv.set_stream_overlap(True)
     ins = [(S.make_logits(w, i, device=DEV), torch.randint(0, w.V, (w.B, w.K), device=DEV, dtype=torch.int32)) for i in range(4)]
     outs = [VerifyBuffers(w.B, w.K, DEV) for _ in ins]
     args = [fv.make_args(w.B, w.K, d, o.accept_len, o.out_tokens, logits=l, state_out=o.state, rollback=o.rollback,
-                         target_argmax=o.target_argmax, entropy=o.entropy, row_flags=o.row_flags)
-            for (l, d), o in zip(ins, outs)]
+                         target_argmax=o.target_argmax, entropy=o.entropy, row_flags=o.row_flags, inputs_ready=i % 2 == 1)
+            for i, ((l, d), o) in enumerate(zip(ins, outs))]
+    torch.cuda.synchronize()
     soak(fv, args, outs, 5000)
     fv.close()
 

@@ -41,7 +41,9 @@ def test_struct_layout_matches_the_header():
     a = Bd.fly_verify_args_t
     assert a.logits.offset == 8 and a.row_stride.offset == 16 and a.draft.offset == 40
     assert a.theta.offset == 48 and a.theta_unit.offset == 56 and a.W.offset == 60 and a.boundary.offset == 64
-    assert a.state_in.offset == 72 and a.row_flags.offset == 128 and a.target_tokens.offset == 136 and C.sizeof(a) == 144
+    assert a.state_in.offset == 72 and a.row_flags.offset == 128 and a.target_tokens.offset == 136
+    assert a.temperature.offset == 144 and a.inputs_ready.offset == 152 and C.sizeof(a) == 160
+    assert C.sizeof(Bd.fly_plan_t) == 32
 
 
 @pytest.mark.parametrize("cfg", [
@@ -83,20 +85,45 @@ def test_header_is_plain_c_and_cxx(tmp_path):
                        check=True)
 
 
-def test_split_planning_rule():
-    # host logic of the logits path: how many pieces a row is cut into (no GPU needed)
-    plan = Bd.lib().fly_verify_plan_splits
-    row = 128256 * 2                                   # one bf16 row of the Llama-3 vocabulary
-    assert plan(148, 144, row, 1) == 1                 # overlapped steps: whole rows
-    assert plan(148, 144, row, 0) == 4                 # a lone grid wants >= 3.5 blocks per SM, evenly
-    assert plan(148, 1088, row, 0) in (1, 2) and plan(148, 2304, 152064 * 2, 0) == 1
-    assert plan(148, 16, row, 0) == 7                  # few rows: as many 32 KB pieces as the row has
-    assert plan(148, 9, 32000 * 4, 0) == 7             # tiny step: down to 16 KB pieces
-    assert plan(148, 16, row, 1) == 3                  # overlapped, few rows: a quarter of the SMs is enough
-    assert plan(0, 1, 1, 0) == 0 and plan(148, 0, row, 0) == 0
-    for rows in (1, 3, 17, 144, 500, 5000):
-        for rb in (64, 4096, 40000, row, 10 * row):
-            for ov in (0, 1):
-                s = plan(148, rows, rb, ov)
-                assert 1 <= s <= 32
-                assert s == 1 or rb // s >= 16384      # pieces never shrink below 16 KB
+def test_launch_geometry_rule():
+    # host logic of the logits path (no GPU needed): how the rows of a step are cut into thread-block ranges
+    row_units = 128256 // 8                                   # 16-byte segments in one bf16 row of the Llama-3 vocabulary
+    p = Bd.plan(148, 144, 128256)
+    assert p.units_per_row == row_units
+    assert p.grid == 144 * 4 and p.slots == 4                 # small step: whole pieces, all resident (4 blocks per SM)
+    assert p.row_span == 4 * p.units_per_block and p.units_per_block * 4 >= row_units
+    p2 = Bd.plan(148, 144, 128256, inputs_ready=True)
+    assert p2.grid == 144 * 2                                 # overlapped steps: two grids resident together
+    big = Bd.plan(148, 1088, 128256)
+    assert big.row_span == row_units and big.grid <= 148 * 4 and big.grid >= 148 * 4 - 4   # large step: rows packed end to end
+    assert Bd.plan(148, 1, 128256).units_per_block >= 1024    # never less than 16 KB per block
+    assert Bd.plan(148, 9, 32000, dtype="f32").grid == 9 * 7
+    L = Bd.lib()
+    out = Bd.fly_plan_t()
+    assert L.fly_verify_plan(0, 1, 128256, Bd.FLY_BF16, 1, 0, 0, out) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_plan(148, 0, 128256, Bd.FLY_BF16, 1, 0, 0, out) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_plan(148, 1, 128256, Bd.FLY_BF16, 1, 0, 0, None) == Bd.FLY_ERR_INVALID_ARG
+    assert L.fly_verify_plan(148, 1, 100, Bd.FLY_BF16, 1, 0, 0, out) == Bd.FLY_ERR_INVALID_ARG   # too short for 16-byte loads
+    for rows in (1, 2, 3, 9, 17, 144, 500, 1088, 2304, 5000, 36864):
+        for vocab, dtype, vec in ((128256, "bf16", True), (152064, "bf16", True), (32000, "f32", True), (257, "bf16", True),
+                                  (1, "f32", False), (7, "bf16", False), (1001, "bf16", False), (1 << 20, "f32", True)):
+            for ready in (False, True):
+                for forced in (0, 1, 2, 5, 32):
+                    p = Bd.plan(148, rows, vocab, dtype, vec, ready, forced)
+                    n, Q, span = p.units_per_row, p.units_per_block, p.row_span
+                    assert Q >= 1 and span >= n and p.grid == -(-(rows * span) // Q) and 1 <= p.slots <= 32
+                    # every row's pieces fit its slots and cover exactly its n units
+                    for r in {0, 1 % rows, rows // 2, rows - 1}:
+                        first, last = (r * span) // Q, (r * span + span - 1) // Q
+                        assert last - first + 1 <= p.slots, (rows, vocab, forced, first, last, p.slots)
+                        covered = 0
+                        for b in range(first, last + 1):
+                            lo = max(b * Q, r * span) - r * span
+                            hi = min((b + 1) * Q, (r + 1) * span) - r * span
+                            covered += max(0, min(hi, n) - min(lo, n))
+                        assert covered == n
+                    if forced:
+                        assert span == min(forced, n, -(-n // Q)) * Q or span % Q == 0
+                        assert span % Q == 0 and span // Q <= forced
+                    elif not ready:
+                        assert p.grid <= max(148 * 4, rows)

@@ -181,3 +181,38 @@ def test_lm_head_logits_is_the_plain_product():
     assert np.array_equal(O.lm_head_logits(e, w)[0], w[5])
     t = torch.matmul(torch.from_numpy(h), torch.from_numpy(w)).numpy()
     assert np.allclose(got, t, rtol=0, atol=1e-12)
+
+
+def test_temperature_divides_the_logits():
+    # Entropy of softmax(l / T).  Pins: T = 1 changes nothing; single spike of height a over a flat row has the
+    # closed form with a / T in place of a; a large T flattens any finite row towards ln V; a small T sharpens a
+    # row with a unique maximum towards 0; the greedy token never moves.
+    V, a = 1000, 6.0
+    row = np.zeros((1, 1, V)); row[0, 0, 123] = a
+    draft = np.zeros((1, 0), dtype=np.int64)
+
+    def closed(h):
+        return math.log(math.exp(h) + V - 1) - h * math.exp(h) / (math.exp(h) + V - 1)
+
+    for T in (0.5, 0.7, 1.0, 1.5, 3.0):
+        r = O.verify_batch(row, draft, theta=1.0, W=0, temperature=T)
+        assert abs(r.entropy[0, 0] - closed(a / T)) < 1e-12 and r.target_argmax[0, 0] == 123
+    rng = np.random.default_rng(5)
+    x = rng.normal(size=(2, 3, 64)) * 4
+    d = np.zeros((2, 2), dtype=np.int64)
+    base = O.verify_batch(x, d, theta=1.0, W=1)
+    same = O.verify_batch(x, d, theta=1.0, W=1, temperature=1.0)
+    assert np.array_equal(base.entropy, same.entropy) and np.array_equal(base.out_tokens, same.out_tokens)
+    hot = O.verify_batch(x, d, theta=1.0, W=1, temperature=1e4)
+    assert np.all(np.abs(hot.entropy - math.log(64)) < 1e-5)
+    cold = O.verify_batch(x, d, theta=1.0, W=1, temperature=1e-3)
+    assert np.all(cold.entropy < 1e-9)
+    for r in (hot, cold):
+        assert np.array_equal(r.target_argmax, base.target_argmax)
+    # scipy on the divided logits (library restatement of the definition)
+    from scipy.special import softmax
+    from scipy.stats import entropy
+    r = O.verify_batch(x, d, theta=1.0, W=1, temperature=0.7)
+    assert np.allclose(r.entropy, entropy(softmax(x / 0.7, axis=-1), axis=-1), atol=1e-12, rtol=0)
+    with pytest.raises(ValueError):
+        O.verify_batch(x, d, theta=1.0, W=1, temperature=0.0)
