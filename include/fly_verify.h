@@ -128,7 +128,14 @@ typedef struct {
   float* entropy;         /* dev [B, K+1] or NULL: H_i in nats (numerator of Eq. 5) */
   uint32_t* row_flags;    /* dev [B, K+1] or NULL: bit 0 non-finite logit (NaN, +inf, or no finite entry);
                              bit 1 draft id outside [0, V) (treated as a mismatch);
-                             bit 2 caller-supplied target token outside [0, V) (mismatch, never deferred) */
+                             bit 2 caller-supplied target token outside [0, V) (mismatch, never deferred);
+                             bit 3 (on position 1 only) the carried state read from state_in is not one this
+                                   library writes (pending outside [0, K], negative rollback_len, or a pending
+                                   window whose correction token is outside [0, V)): it is ignored, i.e. the
+                                   round is verified from the zero state;
+                             bit 4 fused path only: a bounded wait of the GEMM kernel ran out during this step
+                                   (see fly_verify_device_status); set on every row, every position counts as a
+                                   mismatch that is never deferred, so accept_len is 1 and nothing drafted is kept */
 
   /* Optional (NULL = greedy): dev [B, K+1] tokens y_1..y_{K+1} that the caller drew from the target
    * distributions, e.g. by sampling at temperature 1.  The paper's method text defines y_i only as the
@@ -207,7 +214,8 @@ fly_status_t fly_verify_run_partials(fly_verify_t* handle, const fly_verify_args
  * own earlier tokens, n from max_ngram down to min_ngram; at the first n with a match the EARLIEST
  * match position p wins and the tokens that followed it, tokens[p+n .. p+n+K) cut at the sequence end,
  * are proposed.
- *   tokens   dev [B, stride] int32, sequence b holds lengths[b] <= stride tokens
+ *   tokens   dev [B, stride] int32, sequence b holds lengths[b] <= stride tokens (a length outside
+ *            [0, stride] is treated as 0: nothing is proposed, nothing outside the row is read)
  *   draft    dev [B, K]: count[b] proposed tokens, then -1      count  dev [B] (0: no match)
  *   match_pos / match_ngram   dev [B] or NULL: p (-1: none) and n (0: none)
  * 1 <= min_ngram <= max_ngram <= 8.  No handle, no scratch; asynchronous on `cuda_stream`. */
@@ -283,7 +291,9 @@ fly_status_t fly_verify_set_option(fly_verify_t* handle, fly_option_t option, in
  * it and returns without hanging (its outputs are then undefined).  This call
  * synchronises `cuda_stream` and returns FLY_ERR_TIMEOUT if that happened since
  * the last call (the record is cleared), else FLY_OK.  While a record is
- * pending, further fused steps give up early.  Logits-path kernels have no waits. */
+ * pending, further fused steps give up early, and every step run in that state
+ * marks all of its rows with row_flags bit 4, so the failure is also visible in
+ * stream order without a host synchronisation.  Logits-path kernels have no waits. */
 fly_status_t fly_verify_device_status(fly_verify_t* handle, void* cuda_stream);
 
 /* Self-test of that mechanism, safe to run anywhere: enqueues a one-thread kernel that waits, with a

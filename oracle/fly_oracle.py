@@ -35,6 +35,7 @@ import numpy as np
 FLAG_NONFINITE = 1  # a NaN or +inf logit, or a row with no finite logit
 FLAG_BAD_DRAFT = 2  # a draft token id outside [0, V)
 FLAG_BAD_TARGET = 4  # a caller-supplied target token outside [0, V)
+FLAG_BAD_STATE = 8   # (position 1) carried state that the carry extension never writes: ignored
 
 
 def row_stats(x: np.ndarray):
@@ -368,6 +369,13 @@ def verify_batch(logits: np.ndarray, draft: np.ndarray, theta: float, W: int,
             res = verify_round_paper(delta, Hg, th, W, draft[b], y_used[b])
         elif boundary == "carry":
             sin = ZERO_STATE if state_in is None else State(*[int(t) for t in state_in[b]])
+            # The extension only ever writes 0 <= pending <= W <= K, rollback_len >= 0 and, with a window
+            # pending, a correction token inside the vocabulary.  Any other state is not the extension's:
+            # it is flagged on position 1 and the round is verified from the zero state.
+            if sin.pending < 0 or sin.pending > K or sin.rollback_len < 0 or \
+                    (sin.pending > 0 and not (0 <= sin.correction < V)):
+                flags[b, 0] |= FLAG_BAD_STATE
+                sin = ZERO_STATE
             res = verify_round_carry(delta, Hg, th, W, draft[b], y_used[b], sin)
         else:
             raise ValueError(boundary)

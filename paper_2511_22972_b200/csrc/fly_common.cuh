@@ -20,6 +20,8 @@ constexpr int kIdxNone = 0x7fffffff;
 constexpr uint32_t kFlagNonFinite = 1u;
 constexpr uint32_t kFlagBadDraft = 2u;
 constexpr uint32_t kFlagBadTarget = 4u;
+constexpr uint32_t kFlagBadState = 8u;
+constexpr uint32_t kFlagStepFailed = 16u;
 
 // Running state of one (piece of a) row in the base-2 domain.
 //   mx   largest logit seen (raw value; decides the argmax)

@@ -308,7 +308,8 @@ fly_status_t run_fused(fly_verify* h, const fly_verify_args_t* a, cudaStream_t s
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches++;
   }
-  const fly::ScanParams sp = scan_params(h, a, h->lm_folded, 1);
+  fly::ScanParams sp = scan_params(h, a, h->lm_folded, 1);
+  sp.status = h->lm_status;  // a step whose GEMM kernel gave up is marked row by row, in stream order
   e = launch_scan(sp, st);
   if (e != cudaSuccess) return cuda_fail(h, e);
   h->last_launches++;
@@ -341,6 +342,7 @@ fly::ScanParams scan_params(const fly_verify* h, const fly_verify_args_t* a, con
   p.entropy = a->entropy;
   p.row_flags = a->row_flags;
   p.target_tokens = a->target_tokens;
+  p.status = nullptr;
   return p;
 }
 

@@ -15,9 +15,14 @@
 //       reads both halves.  This halves the hidden-state traffic per SM, which is
 //       what bounds a one-CTA version of this kernel (the hidden tile is
 //       re-fetched from L2 for every vocabulary tile).
-//   D = two accumulators of 144 fp32 columns (tensor-memory columns 0..143 and
-//       144..287) in each CTA: lane = one of the CTA's 128 vocabulary entries,
-//       column = position.
+//   D = two accumulators of 144 fp32 columns in each CTA: lane = one of the
+//       CTA's 128 vocabulary entries, column = position.  Tensor memory holds
+//       THREE such slots (columns 0.., 144.., 288..; 432 of 512) and the
+//       accumulators of consecutive tiles rotate through them: accumulator 0 of
+//       the next tile always finds a slot the epilogue is not reading, and
+//       accumulator 1 takes the slot that accumulator 0 of this tile leaves,
+//       which the epilogue drains first - so the tensor pipe does not wait for
+//       the whole epilogue of a tile, only (at most) for its first half.
 // Up to 288 positions need no padding this way (288 = 2 x 144, a legal MMA N),
 // every weight tile meets all positions while it is in shared memory, and the
 // weights (the only large operand) stream from HBM exactly once.
@@ -42,8 +47,9 @@
 // later kernel folds the gridDim.x partials of every row.
 //
 // Every wait on a barrier is bounded: a wait that runs out records a code in
-// *status, and all roles fall through to the common exit (tensor memory is
-// released there).  No TMA load here is a multicast load.
+// *status, and all roles fall through to the common exit (the issuers first let
+// the MMAs they already issued complete; tensor memory is released there).  No
+// TMA load here is a multicast load.
 #pragma once
 #include <cuda.h>
 
@@ -76,12 +82,15 @@ constexpr int kEpiThreads = kEpiWarps * 32;
 constexpr int kWarpW = kEpiWarps, kWarpH = kEpiWarps + 1, kWarpMma = kEpiWarps + 2;  // producers, MMA issuers
 constexpr int kThreads = (kEpiWarps + 4) * 32;
 constexpr int kTmemCols = 512;
+constexpr int kSlots = 3;                           // accumulator slots of kHalfN columns in tensor memory
+static_assert(kSlots * kHalfN <= kTmemCols, "accumulator slots must fit in tensor memory");
+constexpr int kHalfChunks = kHalfN / kChunk;        // 9 blocks of 16 positions per accumulator
 
 constexpr int kOffW = 0;
 constexpr int kOffH = kOffW + kStages * kBytesW;
 constexpr int kOffTurn = kOffH + kStages * kBytesH;
 constexpr int kOffBar = kOffTurn + kTurnBytes;
-constexpr int kNumBars = 2 * kStages + 2;
+constexpr int kNumBars = 2 * kStages + 2 * kSlots + 1;
 constexpr int kOffMisc = kOffBar + kNumBars * 8;
 constexpr int kSmemBytes = kOffMisc + 32 + 1024;    // + slack to align the base to 1024 bytes
 static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
@@ -240,8 +249,11 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   // empty(s), in each CTA: the MMAs that read the stage have completed, the producers may refill it.
   auto full = [&](int s) { return bar0 + 8u * s; };
   auto empty = [&](int s) { return bar0 + 8u * (kStages + s); };
-  const uint32_t tmem_full = bar0 + 8u * (2 * kStages);
-  const uint32_t tmem_empty = tmem_full + 8u;
+  // slot_full(i), in each CTA: the accumulator in tensor-memory slot i is complete.  slot_empty(i), in the leader:
+  // the epilogue threads of both CTAs have read slot i out, the next accumulator may be formed there.
+  auto slot_full = [&](int i) { return bar0 + 8u * (2 * kStages + i); };
+  auto slot_empty = [&](int i) { return bar0 + 8u * (2 * kStages + kSlots + i); };
+  const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 2 * kSlots);  // used only on the give-up path
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + kOffMisc);  // [0] tmem base, [1], [2] go flags of the epilogue groups
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -251,8 +263,11 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
   if (threadIdx.x == 0) {
     const uint32_t issuers = p.n1 > 0 ? 2 : 1;  // one MMA-issuing thread per accumulator
     for (int s = 0; s < kStages; ++s) { mbar_init(full(s), 2); mbar_init(empty(s), issuers); }
-    mbar_init(tmem_full, issuers);
-    mbar_init(tmem_empty, 2 * kEpiThreads);  // the epilogue threads of both CTAs arrive on the leader's
+    for (int i = 0; i < kSlots; ++i) {
+      mbar_init(slot_full(i), 1);                  // the one issuer that formed the accumulator
+      mbar_init(slot_empty(i), 2 * kEpiThreads);   // the epilogue threads of both CTAs arrive on the leader's
+    }
+    mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {  // warp 0 of both CTAs together allocate all of tensor memory (one CTA per SM)
@@ -320,7 +335,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     const int half = warp - kWarpMma;
     if (lane == 0 && rank == 0 && (half == 0 || p.n1 > 0)) {
       const uint32_t idesc = instr_desc(half == 0 ? p.n0 : p.n1, p.w_kmajor != 0);
-      const uint32_t d_tmem = tmem + (uint32_t)(half * kHalfN);
+      const int nh = p.n1 > 0 ? 2 : 1;  // accumulators per tile
       // Everything that changes from one MMA to the next is a 32-bit add: this thread has to issue one
       // MMA every ~70 cycles, so the loop is kept to a few instructions per MMA.
       // A, MN-major: 64-entry chunks lie kBytesWBox apart (leading offset), groups of 8 hidden dims
@@ -335,8 +350,12 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       uint32_t ph = 0;
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
-        // both epilogues must have drained the accumulators of the previous tile
-        if (!mbar_wait(tmem_empty, (t & 1) ^ 1, p.status, kErrTimeoutMma)) break;
+        // this accumulator's slot: the (t * nh + half)-th use of the rotation; the epilogue must have read out
+        // what the slot held three uses ago
+        const int use = t * nh + half;
+        const int slot = use % kSlots;
+        const uint32_t d_tmem = tmem + (uint32_t)(slot * kHalfN);
+        if (!mbar_wait(slot_empty(slot), ((use / kSlots) & 1) ^ 1, p.status, kErrTimeoutMma)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < p.num_kb; ++kb) {
           // TMA-written operands need no tcgen05 fence: the barrier wait orders them before the MMAs
@@ -355,9 +374,16 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
           if (++st == kStages) { st = 0; ph ^= 1; }
         }
         if (ok) {
-          mma_commit(tmem_full);
-          mma_commit(tmem_full + peer_delta);
+          mma_commit(slot_full(slot));
+          mma_commit(slot_full(slot) + peer_delta);
         }
+      }
+      if (!ok) {
+        // Give-up path: MMAs issued before the failed wait may still be reading shared memory and writing
+        // tensor memory.  One more commit to a barrier of its own, and a (bounded) wait on it, lets them
+        // finish before the common exit hands both back.
+        mma_commit(drain_bar);
+        mbar_wait_quiet(drain_bar, 0, 2000000ull);
       }
     }
   } else {
@@ -375,27 +401,41 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
     const int nchunks = (p.R + kChunk - 1) / kChunk;                 // blocks of this launch
     const int my_chunks = nchunks > group ? (nchunks - group + 1) / 2 : 0;  // ... that this group turns
     const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+    const int nh = p.n1 > 0 ? 2 : 1;
+    // the last block of each accumulator that this group turns (-1: none): after reading it the thread hands the
+    // accumulator's slot back
+    int last0 = -1, last1 = -1;
+    for (int k = 0; k < my_chunks; ++k) {
+      if (2 * k + group < kHalfChunks) last0 = k;
+      else last1 = k;
+    }
     for (int t = 0; t < my_tiles; ++t) {
-      if (gtid == 0) misc[1 + group] = mbar_wait(tmem_full, t & 1, p.status, kErrTimeoutEpilogue) ? 1u : 0u;
+      const int use0 = t * nh, use1 = t * nh + 1;
+      const int slot0 = use0 % kSlots, slot1 = use1 % kSlots;
+      if (gtid == 0) {
+        bool okw = mbar_wait(slot_full(slot0), (use0 / kSlots) & 1, p.status, kErrTimeoutEpilogue);
+        if (okw && nh == 2) okw = mbar_wait(slot_full(slot1), (use1 / kSlots) & 1, p.status, kErrTimeoutEpilogue);
+        misc[1 + group] = okw ? 1u : 0u;
+      }
       group_bar(group);
       const bool go = misc[1 + group] != 0;  // one thread per group waits, the group takes the same decision
       if (!go) break;
       tc_fence_after();
       const int v0 = (pair + t * npairs) * kPairV + (int)rank * kBlockV + eighth * 16;
       const int limit = p.V - v0;  // entries of this eighth that exist
-      if (my_chunks == 0) {        // nothing to read for this group: hand the accumulators back at once
-        tc_fence_before();
-        mbar_arrive_remote(map_to_cta(tmem_empty, 0));
-      }
+      // an accumulator of which this group turns no block is handed back at once
+      if (last0 < 0) { tc_fence_before(); mbar_arrive_remote(map_to_cta(slot_empty(slot0), 0)); }
+      if (nh == 2 && last1 < 0) { tc_fence_before(); mbar_arrive_remote(map_to_cta(slot_empty(slot1), 0)); }
 #pragma unroll
       for (int k = 0; k < kGroupChunks; ++k) {
         if (k < my_chunks) {
           const int c = 2 * k + group;
+          const int h = c / kHalfChunks;  // which accumulator the block belongs to
           uint32_t r[16];
-          tmem_ld16(tmem + lane_base + (uint32_t)(c * kChunk), r);
-          if (k == my_chunks - 1) {  // last read of this tile by this thread: hand the accumulators back
+          tmem_ld16(tmem + lane_base + (uint32_t)((h ? slot1 : slot0) * kHalfN + (c - h * kHalfChunks) * kChunk), r);
+          if (k == (h ? last1 : last0)) {  // last read of this accumulator by this thread: hand its slot back
             tc_fence_before();
-            mbar_arrive_remote(map_to_cta(tmem_empty, 0));
+            mbar_arrive_remote(map_to_cta(slot_empty(h ? slot1 : slot0), 0));
           }
           group_bar(group);  // the group is done reading the previous block
 #pragma unroll
@@ -418,7 +458,7 @@ lmhead_verify_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_con
       }
     }
     // Merge the eight vocabulary eighths of every position and write the CTA's partial state.
-    // The weight ring is free by now: every MMA that read it has completed (tmem_full of the last tile).
+    // The weight ring is free by now: every MMA that read it has completed (slot_full of the last tile).
     epi_all_bar();
     Partial* buf = reinterpret_cast<Partial*>(gbase + kOffW);
 #pragma unroll

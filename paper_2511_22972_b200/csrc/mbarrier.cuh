@@ -7,7 +7,11 @@
 
 namespace fly {
 
-constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;  // far above any legitimate wait
+// Far above any legitimate wait (a tile takes ~70 us).  %globaltimer also runs while the context is
+// preempted or time-sliced with another process, so on a shared GPU a wait can in principle run out
+// without a fault in the kernel: the limit is generous for that reason, and a run-out is reported,
+// never trapped on.
+constexpr unsigned long long kWaitLimitNs = 200ull * 1000 * 1000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -51,6 +55,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* st
         return false;
       }
     }
+  }
+  return true;
+}
+
+// The same wait without a status word: for the give-up path, where the failure is already recorded.
+__device__ __forceinline__ bool mbar_wait_quiet(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63) == 0 && global_ns() - t0 > limit_ns) return false;
   }
   return true;
 }

@@ -33,7 +33,10 @@ __global__ void __launch_bounds__(kThreads) pld_draft_kernel(const Params p) {
   __shared__ int found_pos;
   const int b = blockIdx.x;
   const int32_t* tok = p.tokens + (int64_t)b * p.stride;
-  const int L = p.lengths[b];
+  // lengths is device data: a value outside [0, stride] must not steer any load past the sequence's row.
+  // Such a sequence proposes nothing (count 0, match_pos -1), as an empty one does.
+  const int Lraw = p.lengths[b];
+  const int L = (Lraw < 0 || (int64_t)Lraw > p.stride) ? 0 : Lraw;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int pos = -1, ngram = 0;
   for (int n = p.max_ngram; n >= p.min_ngram && pos < 0; --n) {

@@ -43,6 +43,7 @@ struct ScanParams {
   float* entropy;           // [B, K+1] or null
   uint32_t* row_flags;      // [B, K+1] or null
   const int32_t* target_tokens;  // [B, K+1] or null: the caller's y_i instead of the argmax
+  const int* status;             // fused path: device word that is non-zero when a bounded wait of the GEMM kernel ran out
 };
 
 struct RoundOutcome {
@@ -113,10 +114,17 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
     dr[half] = i < K ? p.draft[(int64_t)b * K + i] : 0;
   }
   int pend = 0, len = 0, corr = -1;
+  // A fused step whose GEMM kernel gave up has no usable statistics: every row is flagged, nothing is accepted.
+  const bool failed = p.status != nullptr && *reinterpret_cast<const volatile int*>(p.status) != 0;
+  bool bad_state = false;
   if (p.carry && p.state_in) {
     pend = p.state_in[b * 3 + 0];
     len = p.state_in[b * 3 + 1];
     corr = p.state_in[b * 3 + 2];
+    // The state is device data: only states this library writes are honoured (pending <= W <= K).  Anything
+    // else is flagged and ignored, so that no token id out of range and no negative count can leave here.
+    bad_state = pend < 0 || pend > K || len < 0 || (pend > 0 && (corr < 0 || corr >= p.V));
+    if (bad_state) { pend = 0; len = 0; corr = -1; }
   }
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
@@ -138,6 +146,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
       const float H = fmaxf(kLn2 * (log2f(acc.S) - acc.u / acc.S), 0.f);
       uint32_t flag = 0;
       if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx <= kMaskFloor) flag |= kFlagNonFinite;
+      if (failed) flag |= kFlagStepFailed;
       int y = acc.idx;
       if (flag || y < 0 || y >= p.V) y = 0;  // keep every emitted id in range
       const int greedy = y;
@@ -154,7 +163,7 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
       }
       if (p.target_argmax) p.target_argmax[row] = greedy;
       if (p.entropy) p.entropy[row] = H;
-      if (p.row_flags) p.row_flags[row] = flag;
+      if (p.row_flags) p.row_flags[row] = flag | ((i == 0 && bad_state) ? kFlagBadState : 0u);
     }
     const uint64_t mb = __ballot_sync(0xffffffffu, is_mism);
     const uint64_t db = __ballot_sync(0xffffffffu, is_defer);

@@ -13,10 +13,11 @@ def oracle_entropy(rows: torch.Tensor):
     return O.row_stats(rows.double().cpu().numpy())[0]
 
 
-def draw(w, step=0, setting=0, device="cuda", thetas=None, guard=True):
-    """Logits (entropies kept >= 1e-3 away from every threshold) and drafts."""
+def draw(w, step=0, setting=0, device="cuda", thetas=None, guard=True, temperature=1.0):
+    """Logits (entropies - at the given temperature - kept >= 1e-3 away from every threshold) and drafts."""
+    ent = oracle_entropy if temperature == 1.0 else (lambda rows: O.row_stats(rows.double().cpu().numpy() / temperature)[0])
     logits = S.make_logits(w, step, device=device, setting=setting,
-                           entropy_fn=oracle_entropy if guard else None,
+                           entropy_fn=ent if guard else None,
                            theta_nats=thetas if thetas is not None else w.theta)
     top5 = S.rank5(logits.view(-1, w.V))
     draft = S.make_draft(w, step, top5, setting=setting)

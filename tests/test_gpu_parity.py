@@ -421,3 +421,51 @@ def test_many_sequences_and_a_very_long_vocabulary():
     out = gpu_step(fv, logits, draft, 1.0, 1)
     assert out.target_argmax.view(-1)[1].item() == 0
     assert abs(out.entropy.view(-1)[1].item() - math.log(V)) < 1e-4
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 128256), ("f32", 32000), ("bf16", 1001)])
+@pytest.mark.parametrize("T", [0.7, 1.0, 1.5, 4.0])
+def test_temperature_scaled_entropy(dtype, V, T):
+    # the entropy of softmax(l / T): 1/T is folded into the exponent constant of every kernel and merge
+    w = small(dtype, B=5, K=6, V=V)
+    fv = FlyVerify(w.B, w.K, V, dtype)
+    logits, draft = draw(w, step=int(T * 10), temperature=T)
+    for splits in (0, 3):
+        fv.set_splits(splits)
+        err, out, ref = check(fv, logits, draft, w.theta, 2, temperature=T, what=f"{dtype} V={V} T={T} splits={splits}")
+    plain = oracle_step(logits, draft, w.theta, 2)
+    assert np.array_equal(ref.target_argmax, plain.target_argmax)          # the greedy token does not depend on T
+    if T != 1.0:
+        assert np.abs(ref.entropy - plain.entropy).max() > 1e-2           # ... the entropy does
+    check(fv, logits.cpu().pin_memory(), draft.cpu().pin_memory(), w.theta, 2, temperature=T, host=True, what="host buffers")
+    check(fv, logits, draft, 0.3, 2, theta_unit="normalized", temperature=T, what="normalised threshold")
+    fv.close()
+
+
+def test_temperature_argument_range():
+    from paper_2511_22972_b200 import VerifyBuffers, binding as Bd
+    w = small("bf16", B=1, K=2, V=1024)
+    fv = FlyVerify(1, 2, 1024, "bf16")
+    logits, draft = draw(w, guard=False)
+    out = VerifyBuffers(1, 2, DEV)
+    for T in (-1.0, 1e-9, 1e9, float("nan"), float("inf")):
+        a = fv.make_args(1, 2, draft, out.accept_len, out.out_tokens, logits=logits, state_out=out.state, temperature=T)
+        with pytest.raises(Bd.FlyError) as e:
+            fv.run(a)
+        assert e.value.status == Bd.FLY_ERR_INVALID_ARG
+    a = fv.make_args(1, 2, draft, out.accept_len, out.out_tokens, logits=logits, state_out=out.state)
+    a.inputs_ready = 2
+    with pytest.raises(Bd.FlyError):
+        fv.run(a)
+
+
+def test_carried_state_that_the_library_never_writes_is_flagged_and_ignored():
+    w = small("bf16", B=8, K=4, V=4096, boundary="carry")
+    fv = FlyVerify(w.B, w.K, w.V, "bf16")
+    logits, draft = draw(w, step=2)
+    state = [[0, 0, -1], [5, 2, 1], [-1, 2, 1], [1, -3, 1], [2, 2, 4096], [1, 2, -1], [2, 3, 17], [4, 9, 4095]]
+    err, out, ref = check(fv, logits, draft, 1.0, 3, boundary="carry", state=state, what="bad carried state")
+    flags = out.row_flags.cpu().numpy()
+    assert (flags[[1, 2, 3, 4, 5], 0] & 8).all() and not (flags[[0, 6, 7], 0] & 8).any()
+    toks = out.out_tokens.cpu().numpy()
+    assert toks.max() < w.V and toks.min() >= -1 and (out.rollback.cpu().numpy() >= 0).all()

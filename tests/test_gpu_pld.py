@@ -60,3 +60,18 @@ def test_argument_errors():
         with pytest.raises(Bd.FlyError) as e:
             Bd.pld_draft(t, l, K, mx, mn)
         assert e.value.status == Bd.FLY_ERR_INVALID_ARG
+
+
+def test_lengths_outside_the_row_propose_nothing_and_read_nothing_outside_it():
+    # lengths is device data: a length larger than the row stride, or negative, must not steer a load past the row
+    B, stride, K = 6, 64, 8
+    rng = random.Random(3)
+    tok = torch.tensor([[rng.randrange(4) for _ in range(stride)] for _ in range(B)], dtype=torch.int32)
+    lengths = torch.tensor([stride, stride + 1, 10 ** 9, -1, -(10 ** 9), 40], dtype=torch.int32)
+    draft, count, pos, ng = Bd.pld_draft(tok.to(DEV), lengths.to(DEV), K, 3, 1, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for b in (1, 2, 3, 4):
+        assert count[b].item() == 0 and pos[b].item() == -1 and ng[b].item() == 0 and (draft[b] == -1).all()
+    for b in (0, 5):
+        prop, p, n = oracle_pld(tok[b, :lengths[b]].tolist(), K, 3, 1)
+        assert count[b].item() == len(prop) and pos[b].item() == p and draft[b, :len(prop)].tolist() == prop

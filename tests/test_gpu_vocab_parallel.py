@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def sharded_step(w, logits, draft, world, theta, W, theta_unit="nats", boundary="reject", state=None):
+def sharded_step(w, logits, draft, world, theta, W, theta_unit="nats", boundary="reject", state=None, temperature=0.0):
     B, K1, V = logits.shape
     rows = B * K1
     flat = logits.view(rows, V)
@@ -25,7 +25,7 @@ def sharded_step(w, logits, draft, world, theta, W, theta_unit="nats", boundary=
         off, width = D.shard_vocab(V, D.Ranks(rank, world, 0, ""))
         fv = FlyVerify(B, K1 - 1, max(width, 1), w.dtype)
         if width > 0:
-            fv.reduce_shard(flat[:, off:off + width], off, gathered[rank], st)
+            fv.reduce_shard(flat[:, off:off + width], off, gathered[rank], st, temperature=temperature)
         else:                                                     # an empty slice contributes the empty state
             gathered[rank] = torch.tensor([-999424.0, 0.0, 0.0, 0.0])
             gathered[rank].view(torch.int32)[:, 3] = 0x7fffffff
@@ -37,7 +37,7 @@ def sharded_step(w, logits, draft, world, theta, W, theta_unit="nats", boundary=
     a = merger.make_args(B, K1 - 1, draft, out.accept_len, out.out_tokens, theta=theta, theta_unit=theta_unit, W=W,
                          boundary=boundary, state_in=out.state if boundary == "carry" else None, state_out=out.state,
                          rollback=out.rollback, target_argmax=out.target_argmax, entropy=out.entropy,
-                         row_flags=out.row_flags)
+                         row_flags=out.row_flags, temperature=temperature)
     merger.run_partials(a, gathered, world, V, st)
     torch.cuda.synchronize()
     return out
@@ -83,3 +83,12 @@ def test_carry_state_with_sharded_vocabulary():
     state = [[b % 3, 4, 11] for b in range(w.B)]
     out = sharded_step(w, logits, draft, 2, w.theta, w.W, boundary="carry", state=state)
     assert_parity(out, oracle_step(logits, draft, w.theta, w.W, "carry", state), "carry tp2")
+
+
+@pytest.mark.parametrize("T", [0.7, 1.5])
+def test_sharded_vocabulary_at_a_temperature(T):
+    # every rank and the merging call pass the same temperature: the merged entropy is that of softmax(l / T)
+    w = S.shrink(S.LLAMA3, B=3, K=5, V=50264)
+    logits, draft = draw(w, step=5, temperature=T)
+    out = sharded_step(w, logits, draft, 4, 1.0, 2, temperature=T)
+    assert_parity(out, oracle_step(logits, draft, 1.0, 2, temperature=T), f"tp4 T={T}")

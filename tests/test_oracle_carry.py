@@ -135,3 +135,23 @@ def test_verify_batch_carry_chain_shapes():
     r2 = O.verify_batch(lg, d2, 1.0, W, boundary="carry", state_in=r.state_out)
     assert r2.accept_len.tolist() == [1, 3] and r2.rollback.tolist() == [2, 0]
     assert r2.out_tokens.tolist() == [[1, -1, -1], [0, 1, 2]]
+
+
+def test_a_state_the_extension_never_writes_is_flagged_and_ignored():
+    # V = 4, K = 3, flat rows (Defer everywhere, argmax 0), drafts all 0: an accept-all round from the zero state.
+    # A carried state is only honoured if it is one the extension can have written: 0 <= pending <= K,
+    # rollback_len >= 0, and a correction inside the vocabulary while a window is pending.
+    x = np.zeros((1, 4, 4))
+    d = np.array([[0, 0, 0]])
+    for bad in ([4, 2, 1], [-1, 2, 1], [1, -3, 1], [2, 2, 9], [1, 2, -1]):
+        r = O.verify_batch(x, d, theta=0.0, W=1, boundary="carry", state_in=np.array([bad]))
+        assert r.row_flags.tolist() == [[O.FLAG_BAD_STATE, 0, 0, 0]], bad
+        assert r.accept_len.tolist() == [4] and r.rollback.tolist() == [0] and r.out_tokens.tolist() == [[0, 0, 0, 0]]
+        assert r.state_out.tolist() == [[0, 0, -1]]
+    # a legal pending state is used: position 1 mismatches (draft 2 against argmax 0) and revokes it
+    r = O.verify_batch(x, np.array([[2, 0, 0]]), theta=0.0, W=1, boundary="carry", state_in=np.array([[1, 2, 3]]))
+    assert r.row_flags.tolist() == [[0, 0, 0, 0]] and r.accept_len.tolist() == [1] and r.rollback.tolist() == [2]
+    assert r.out_tokens.tolist() == [[3, -1, -1, -1]]
+    # with nothing pending the correction field is not looked at (the zero state carries -1 there)
+    r = O.verify_batch(x, d, theta=0.0, W=1, boundary="carry", state_in=np.array([[0, 0, -1]]))
+    assert r.row_flags.tolist() == [[0, 0, 0, 0]]

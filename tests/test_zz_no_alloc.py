@@ -7,25 +7,22 @@ This file is collected last on purpose: it is an addition outside the paper's
 method, and a failure here must not hide the result of any other test.
 
 The check: two calls in a row through the C ABI, different shapes, each
-compared with what the handle-based entry point (fly_verify_run) writes for the
-same inputs - integers bit for bit, entropy within the tolerance of the parity
-tests.  Nothing here depends on what ran before in the process: the entry point
-clears its arrival counters itself and both calls are on one stream.
+compared with the fp64 oracle (the same comparison as every parity test) and,
+as a second check, with what the handle-based entry point (fly_verify_run)
+writes for the same inputs - integers bit for bit, entropy within the tolerance
+of the parity tests.  Nothing here depends on what ran before in the process:
+the entry point clears its arrival counters itself and both calls are on one
+stream.
 """
 import pytest
 import torch
 
 from paper_2511_22972_b200 import FlyError, FlyVerify, VerifyBuffers, binding as Bd, synthetic as S
+from tests._parity import assert_parity, draw, oracle_step
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
 ENTROPY_TOL = 1e-4
-
-
-def _inputs(w, step):
-    logits = S.make_logits(w, step, device=DEV)
-    draft = S.make_draft(w, step, S.rank5(logits.view(-1, w.V)))
-    return logits, draft
 
 
 def _args(w, logits, draft, out, boundary, state_in):
@@ -48,7 +45,7 @@ def test_static_entry_point_matches_the_handle_entry_point_twice_in_a_row():
         (S.shrink(S.SERVING, B=40, K=5, V=50264), "carry"),        # more sequences, carried state, other vocab
     ]
     for n, (w, boundary) in enumerate(cases):
-        logits, draft = _inputs(w, step=11 + n)
+        logits, draft = draw(w, step=11 + n)                       # entropies kept away from the threshold
         carry = boundary == "carry"
         state0 = torch.tensor([[1, 3, 7]] * w.B, dtype=torch.int32, device=DEV) if carry else None
 
@@ -67,6 +64,8 @@ def test_static_entry_point_matches_the_handle_entry_point_twice_in_a_row():
             getattr(got, name).fill_(-7)                           # stale values must all be overwritten
         Bd.run_static(_args(w, logits, draft, got, boundary, got.state if carry else None), w.V, w.dtype, 0, st)
         torch.cuda.synchronize()
+        oracle = oracle_step(logits, draft, w.theta, w.W, boundary, state0.cpu().numpy() if carry else None)
+        assert_parity(got, oracle, f"call {n + 1} ({w.name}) against the oracle")
         _same(got, ref, f"call {n + 1} ({w.name})")
         s = got.accept_len.cpu()
         assert bool(((s >= 1) & (s <= w.K + 1)).all())
