@@ -50,10 +50,12 @@ MIN_TIMED_S = 0.05                 # every timed region lasts at least this long
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (bytes), keyed by kernel; None where the kernel has changed since its counters were taken.
 NCU_TRAFFIC = {
-    # reduce_rows_flat, long_draft_batch (1088 rows x 128256 bf16): see profiles/reduce_rows_flat_long_draft_batch.md
-    "reduce_rows_flat": None,
-    # lmhead_verify_kernel at V = 64000: see profiles/lmhead_verify_kernel_fused_lm_head.md
-    "lmhead_verify_kernel": None,
+    # reduce_rows_flat, long_draft_batch (279,085,056 algorithmic bytes): 279.15 MB read + 6.00 MB written
+    # (profiles/reduce_rows_flat_long_draft_batch.md); scaled to other workloads by their algorithmic bytes
+    "reduce_rows_flat": {"bytes": 285.16e6, "units": 279085056},
+    # lmhead_verify_kernel at V = 64000: 1.0675 GB read + 4.9 MB written (profiles/lmhead_verify_kernel_fused_lm_head.md);
+    # scaled by V
+    "lmhead_verify_kernel": {"bytes": 1.0724e9, "units": 64000},
 }
 
 
@@ -206,7 +208,7 @@ def build_inputs(w, device, nbuf, near_miss=True):
     return bufs
 
 
-def bench_logits(w, ranks, device, steps, warmup, launch, peaks, near_miss=True):
+def bench_logits(w, ranks, device, steps, warmup, launch, peaks, near_miss=True, splits=0):
     """One logits-path workload: serial (plain stream order) and overlapped (inputs_ready) step times."""
     import torch
     from paper_2511_22972_b200 import FlyVerify, VerifyBuffers
@@ -215,6 +217,7 @@ def bench_logits(w, ranks, device, steps, warmup, launch, peaks, near_miss=True)
     bufs = build_inputs(w, device, nbuf, near_miss)
     out = VerifyBuffers(w.B, w.K, device)
     fv = FlyVerify(w.B, w.K, w.V, w.dtype, device=ranks.local_rank)
+    fv.set_splits(splits)
     carry = w.boundary == "carry"
 
     def mk(l, d, ready):
@@ -596,7 +599,7 @@ def run_vocab_parallel(args, w):
                      "peak": peaks["hbm"], "peak_kind": f"of {peaks['kind']}", "unit": "GB/s", "frac": achieved / peaks["hbm"],
                      "bytes_per_launch": slice_bytes, "us_per_launch": ms * 1e3,
                      "note": "duration = whole step: slice reduction + fold + all-gather + merge + acceptance scan",
-                     "traffic": ncu_traffic("reduce_rows_flat", w.rows * width)},
+                     "traffic": ncu_traffic("reduce_rows_flat", w.rows * width * w.elem_bytes)},
         "e2e": None,
         "gpu_launches": 4 * n,
         "clocks": clk.summary(),
@@ -685,6 +688,8 @@ def main():
                     help="logits path: launch the timed steps from CUDA graphs (default) or one by one from the host")
     ap.add_argument("--shard", default="batch", choices=["batch", "vocab"])
     ap.add_argument("--no-extra", action="store_true", help="time only --workload (no `workloads` object)")
+    ap.add_argument("--splits", type=int, default=0, help="logits path: cut every row into exactly this many pieces "
+                    "(FLY_OPT_SPLITS; 0 = the library's own choice); recorded in config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--vocab", type=int, default=None, help="run the workload's recipe at another vocabulary size "
                     "(smaller cases for profiler captures); recorded in config")
@@ -717,7 +722,7 @@ def main():
     peaks = measured_peaks()
 
     # ---- the named workload: whole steps over device-resident inputs, serial and overlapped ---------------
-    r = bench_logits(w, ranks, device, args.steps, warmup, args.launch, peaks)
+    r = bench_logits(w, ranks, device, args.steps, warmup, args.launch, peaks, splits=args.splits)
     assert r["launches_per_step"] == 1, r["launches_per_step"]     # the acceptance scan is the tail of the reduction
     ms_per_step = r["serial_ms"]
     rows_all = w.rows * ranks.world
@@ -730,7 +735,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": w.B, "K": w.K, "V": w.V, "logits_dtype": w.dtype,
                    "theta_nats": w.theta, "W": w.W, "boundary": w.boundary, "parallelism": f"dp{ranks.world}",
-                   "launch": args.launch, "order": "plain stream order (each step waits for the previous kernel before its first read)",
+                   "launch": args.launch, "splits": args.splits or "auto", "order": "plain stream order (each step waits for the previous kernel before its first read)",
                    "l2": f"inputs rotate over {r['nbuf']} distinct buffers = {r['nbuf'] * r['step_bytes'] / 1e6:.0f} MB (> 2x L2)"},
         "hbm_gbs": rows_all * w.V * w.elem_bytes / (ms_per_step * 1e-3) / 1e9,
         "hbm_pct_of_peak": 100.0 * achieved / peaks["hbm"],

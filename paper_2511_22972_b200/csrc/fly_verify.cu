@@ -91,6 +91,7 @@ struct FlatPlan {
   int64_t span = 1;   // units a row takes in the flat index space
   int grid = 1;
   int slots = 1;
+  int pieces = 0;     // > 0: every row is cut into exactly this many pieces (span = pieces * Q)
 };
 // stride_units: units one thread block covers per loop iteration (all its warps, one slice each).
 FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int64_t stride_units, int cap,
@@ -128,6 +129,7 @@ FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int
     if (s > 1) pl.Q = (pl.Q + 7) / 8 * 8;        // pieces start on 128-byte boundaries of the row
     s = (n + pl.Q - 1) / pl.Q;                   // pieces that are not empty
     pl.span = s * pl.Q;
+    pl.pieces = (int)s;
   }
   const int64_t total = rows * pl.span;
   pl.grid = (int)((total + pl.Q - 1) / pl.Q);
@@ -149,6 +151,29 @@ void fill_launch(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, unsigned gr
   cfg->numAttrs = 1;
 }
 
+// Shared memory of the row reduction's cp.async rings (vector path), per block.
+constexpr int kReduceRingBytes = fly::kReduceWarps * fly::kDepth * kReduceUnroll * 32 * 16;
+
+// Function attributes are per device: set them once on every device that launches the row reduction.
+// The rings of all resident blocks only fit on an SM whose L1/shared split favours shared memory.
+constexpr int kMaxDevices = 64;
+void ensure_reduce_attrs(int device) {
+  static std::mutex mu;
+  static bool done[kMaxDevices] = {};
+  if (device >= 0 && device < kMaxDevices) {
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[device]) return;
+    done[device] = true;
+  }
+  auto set = [](auto kernel) {
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kReduceRingBytes);
+    cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+  };
+  set(fly::reduce_rows_flat<__nv_bfloat16, kReduceUnroll, true>);
+  set(fly::reduce_rows_flat<float, kReduceUnroll, true>);
+  (void)cudaGetLastError();
+}
+
 template <typename T>
 bool vector_path_ok(const void* logits, int64_t row_stride, int V) {
   return ((reinterpret_cast<uintptr_t>(logits) & 15u) == 0) && ((row_stride * (int64_t)sizeof(T)) % 16 == 0) &&
@@ -168,7 +193,8 @@ cudaError_t launch_reduce(int sm_count, const void* logits, int64_t row_stride, 
   const int64_t stride_units = (int64_t)fly::kReduceWarps * kReduceUnroll * 32;
   const FlatPlan pl = plan_flat(sm_count, rows, n, min_units, stride_units, cap, inputs_ready, forced);
   fly::ReducePlan g;
-  g.n = n; g.span = pl.span; g.Q = pl.Q; g.total = rows * pl.span; g.slots = pl.slots; g.V = V; g.row_stride = row_stride;
+  g.n = n; g.span = pl.span; g.Q = pl.Q; g.total = rows * pl.span; g.slots = pl.slots;
+  g.pieces = pl.Q < (1 << 30) ? pl.pieces : 0; g.V = V; g.row_stride = row_stride;
   g.scale = scale; g.wait_first = inputs_ready ? 0 : 1;
   tail->splits = pl.slots;
   tail->units_per_row = n;
@@ -178,16 +204,7 @@ cudaError_t launch_reduce(int sm_count, const void* logits, int64_t row_stride, 
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
   fill_launch(&cfg, attr, (unsigned)pl.grid, fly::kReduceThreads, st, true);
-  // The rings of all resident blocks only fit on an SM whose L1/shared split favours shared memory.
-  constexpr int kRingBytes = fly::kReduceWarps * fly::kDepth * kReduceUnroll * 32 * 16;
-  static std::once_flag ring_once;
-  std::call_once(ring_once, [] {
-    cudaFuncSetAttribute(fly::reduce_rows_flat<T, kReduceUnroll, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
-    cudaFuncSetAttribute(fly::reduce_rows_flat<T, kReduceUnroll, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                         cudaSharedmemCarveoutMaxShared);
-    (void)cudaGetLastError();
-  });
-  cfg.dynamicSmemBytes = vec ? kRingBytes : 0;
+  cfg.dynamicSmemBytes = vec ? kReduceRingBytes : 0;
   if (vec)
     return cudaLaunchKernelEx(&cfg, fly::reduce_rows_flat<T, kReduceUnroll, true>, static_cast<const T*>(logits), g, partials,
                               *tail);
@@ -195,9 +212,11 @@ cudaError_t launch_reduce(int sm_count, const void* logits, int64_t row_stride, 
                             *tail);
 }
 
-cudaError_t launch_reduce_any(fly_dtype_t dt, int sm_count, const void* logits, int64_t row_stride, int V, int64_t rows,
-                              int forced, int cap, fly::Partial* partials, cudaStream_t st, fly::ScanParams* tail,
-                              float scale, bool inputs_ready) {
+// The current device must be the one the pointers belong to (its ordinal is `device`).
+cudaError_t launch_reduce_any(int device, fly_dtype_t dt, int sm_count, const void* logits, int64_t row_stride, int V,
+                              int64_t rows, int forced, int cap, fly::Partial* partials, cudaStream_t st,
+                              fly::ScanParams* tail, float scale, bool inputs_ready) {
+  ensure_reduce_attrs(device);
   if (dt == FLY_BF16)
     return launch_reduce<__nv_bfloat16>(sm_count, logits, row_stride, V, rows, forced, cap, partials, st, tail, scale,
                                         inputs_ready);
@@ -489,7 +508,7 @@ fly_status_t fly_verify_reduce_shard(fly_verify_t* h, int32_t rows, const void* 
   const float scale = exponent_scale(temperature);
   fly::ScanParams none;
   memset(&none, 0, sizeof(none));  // tickets == NULL: no acceptance scan in this launch
-  cudaError_t e = launch_reduce_any(h->cfg.logits_dtype, h->sm_count, logits, stride, V, rows, h->forced_splits, kMaxSplits,
+  cudaError_t e = launch_reduce_any(h->cfg.device, h->cfg.logits_dtype, h->sm_count, logits, stride, V, rows, h->forced_splits, kMaxSplits,
                                     h->partials, st, &none, scale, false);
   if (e != cudaSuccess) return cuda_fail(h, e);
   cudaLaunchConfig_t cfg;
@@ -616,9 +635,12 @@ fly_status_t fly_verify_run(fly_verify_t* h, const fly_verify_args_t* a, void* c
   if (!a->logits) return run_fused(h, a, st);
 
   fly::ScanParams p = scan_params(h, a, h->partials, 1);
+  // The acceptance scan runs as the tail of the reduction (the block that completes a sequence verifies it) unless
+  // the handle asks for a kernel of its own.  Measured in plain stream order the two cost the same; the tail also
+  // lets consecutive steps overlap (inputs_ready) and keeps a step at one launch.
   const bool fused_tail = h->scan_mode == 0;
   p.tickets = fused_tail ? h->tickets : nullptr;
-  cudaError_t e = launch_reduce_any(h->cfg.logits_dtype, h->sm_count, a->logits, stride, V, rows, h->forced_splits,
+  cudaError_t e = launch_reduce_any(h->cfg.device, h->cfg.logits_dtype, h->sm_count, a->logits, stride, V, rows, h->forced_splits,
                                     kMaxSplits, h->partials, st, &p, p.scale, a->inputs_ready != 0);
   if (e != cudaSuccess) return cuda_fail(h, e);
   h->last_launches++;
@@ -804,7 +826,7 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
   // The arrival counters must start at zero, whatever an earlier call left behind.
   cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)a->B * 4, st);
   if (e != cudaSuccess) return FLY_ERR_CUDA;
-  e = launch_reduce_any(logits_dtype, h.sm_count, a->logits, stride, vocab, rows, 0, cap, partials, st, &p, p.scale,
+  e = launch_reduce_any(device, logits_dtype, h.sm_count, a->logits, stride, vocab, rows, 0, cap, partials, st, &p, p.scale,
                         a->inputs_ready != 0);
   return e == cudaSuccess ? FLY_OK : FLY_ERR_CUDA;
 }

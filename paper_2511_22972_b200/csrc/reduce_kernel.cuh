@@ -292,6 +292,7 @@ struct ReducePlan {
   int64_t span;    // units a row takes in the flat index space (>= n)
   int64_t Q;       // units per block
   int64_t total;   // rows * span
+  int pieces;      // > 0: span = pieces * Q, block b is piece b % pieces of row b / pieces (32-bit arithmetic)
   int slots;       // Partial slots per row (>= the largest number of pieces of any row)
   int V;
   int64_t row_stride;  // elements
@@ -350,15 +351,12 @@ __device__ __forceinline__ void sequence_tail(const ScanParams& p, int row, unsi
   if (lane == 0) {
     const unsigned t = atomicAdd(p.tickets + b, units);
     last = (t + units == (unsigned)K1 * (unsigned)p.units_per_row);
-    if (last) {
-      p.tickets[b] = 0;  // ready for the next launch
-      __threadfence();
-    }
   }
   last = __shfl_sync(0xffffffffu, last, 0);
   if (last) {
     __threadfence();  // every lane reads the other blocks' partials after the ticket was seen
     scan_one_sequence(p, b, lane, sm_y);
+    if (lane == 0) p.tickets[b] = 0;  // ready for the next launch (ordered by the end of this kernel; off the critical path)
   }
 }
 
@@ -396,15 +394,24 @@ reduce_rows_flat(const T* __restrict__ logits, const __grid_constant__ ReducePla
   // grid's completion before it touches anything this grid writes.
   asm volatile("griddepcontrol.launch_dependents;");
 
-  const int64_t f0 = (int64_t)blockIdx.x * g.Q;
-  const int64_t f_end = min(f0 + g.Q, g.total);
-  int row = (int)(f0 / g.span);
-  int u0 = (int)(f0 - (int64_t)row * g.span);                              // first unit of this block's piece inside the row
-  int slot = (int)((int64_t)blockIdx.x - ((int64_t)row * g.span) / g.Q);   // pieces of the row that earlier blocks hold
-  int u1 = (int)min(g.n, (int64_t)u0 + (f_end - f0));                      // end of the piece inside the row
-  // flat units of this block not yet assigned to a piece (a row ends at its span, not at n)
-  int64_t left = f_end - f0;
-  int64_t take = min((int64_t)g.span - u0, left);                          // flat units the current piece takes
+  int row, u0, u1, slot;  // the current piece: units [u0, u1) of `row`, stored in the row's slot `slot`
+  int64_t left, take;     // flat units of this block not yet assigned to a piece; flat units the current piece takes
+  if (g.pieces > 0) {     // whole pieces of rows: one per block, 32-bit arithmetic (the common small-step case)
+    row = (int)blockIdx.x / g.pieces;
+    slot = (int)blockIdx.x - row * g.pieces;
+    u0 = slot * (int)g.Q;
+    u1 = min((int)g.n, u0 + (int)g.Q);
+    left = take = g.Q;
+  } else {
+    const int64_t f0 = (int64_t)blockIdx.x * g.Q;
+    const int64_t f_end = min(f0 + g.Q, g.total);
+    row = (int)(f0 / g.span);
+    u0 = (int)(f0 - (int64_t)row * g.span);
+    slot = (int)((int64_t)blockIdx.x - ((int64_t)row * g.span) / g.Q);     // pieces of the row that earlier blocks hold
+    u1 = (int)min(g.n, (int64_t)u0 + (f_end - f0));
+    left = f_end - f0;                                                     // (a row ends at its span, not at n)
+    take = min((int64_t)g.span - u0, left);
+  }
 
   // Copy side of the pipeline.  A warp's slices of the piece [pu0, pu1) of the row at `prow` start at
   // ps = pu0 + warp * kSlice and lie kStride apart; issue() copies the next one into a ring stage.
