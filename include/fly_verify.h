@@ -250,7 +250,7 @@ fly_status_t fly_pld_draft(int32_t device, int32_t B, const int32_t* tokens, int
  * The first call on each device looks up the device address of the built-in
  * array (which also makes the CUDA runtime load the library's device code).
  * Make that first call outside any stream capture; later calls only enqueue
- * work on `cuda_stream` (one 4 KB memset of the arrival counters, one kernel).
+ * work on `cuda_stream` (one memset of the B arrival counters, one kernel).
  *
  * All calls on a device share the one array, and it keeps whatever the last
  * call left there.  The counters are cleared on the stream at the start of
