@@ -257,21 +257,25 @@ def logits_row(w, r, peaks, world):
     }
 
 
-def h2d_bandwidth(device, nbytes, stream):
-    """Pinned host -> device copy bandwidth for a buffer of nbytes (GB/s), best of 5: what bounds `e2e`."""
+def h2d_bandwidth(device, nbytes, stream, copies=20):
+    """Pinned host -> device copy bandwidth for buffers of nbytes (GB/s): `copies` back-to-back copies timed as a
+    whole, best of 3 such batches.  This is what bounds `e2e`, whose every step makes one such copy."""
     import torch
     n = max(int(nbytes), 1 << 20)
     src = torch.empty(n, dtype=torch.uint8).pin_memory()
     dst = torch.empty(n, dtype=torch.uint8, device=device)
     best = 0.0
     with torch.cuda.stream(stream):
-        for _ in range(6):
+        dst.copy_(src, non_blocking=True)
+        stream.synchronize()
+        for _ in range(3):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            dst.copy_(src, non_blocking=True)
+            for _ in range(copies):
+                dst.copy_(src, non_blocking=True)
             e1.record(stream)
             stream.synchronize()
-            best = max(best, n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+            best = max(best, copies * n / (e0.elapsed_time(e1) * 1e-3) / 1e9)
     return best
 
 

@@ -79,11 +79,7 @@ fly_status_t cuda_fail(fly_verify* h, cudaError_t e) {
   return FLY_ERR_CUDA;
 }
 
-// Launch geometry of the row reduction (the flat partition described at the head of reduce_kernel.cuh).
-// The grid should be resident all at once and give every block the same number of bytes: blocks then
-// finish together, whatever the number of rows, and a grid that runs alone has no ragged last wave.
-//   gmax   blocks that fit on the device at once (half of them when consecutive steps are meant to
-//          overlap, so that two grids can be resident together)
+// Launch geometry of the row reduction (the flat index space described at the head of reduce_kernel.cuh).
 //   n      units per row, min_units: a block should not get less than this
 //   cap    Partial slots available per row (>= 1)
 struct FlatPlan {
@@ -93,30 +89,41 @@ struct FlatPlan {
   int slots = 1;
   int pieces = 0;     // > 0: every row is cut into exactly this many pieces (span = pieces * Q)
 };
-// stride_units: units one thread block covers per loop iteration (all its warps, one slice each).
+// Launch shape.  Measured on the bench workloads (144 .. 2304 rows of 250 - 300 KB): whole pieces of rows, one per
+// block, are at least as fast as packed rows whenever they fill the resident slots reasonably well - a row boundary
+// inside a block drains that block's copy ring once, and the hardware scheduler back-fills a second wave well.
+//   plain stream order   pieces per row so that the grid just fits on the device at once (4 blocks per SM);
+//                        more rows than slots: whole rows, several waves
+//   inputs_ready         about one block per SM: consecutive steps then overlap four deep, which hides each
+//                        step's ramp and its hand-off tail behind its neighbours' streaming
+//   packed rows          only where whole pieces would leave more than a quarter of the last wave's slots empty
 FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int64_t stride_units, int cap,
                    bool inputs_ready, int forced) {
+  (void)stride_units;
   FlatPlan pl;
-  const int bps = inputs_ready ? fly::kReduceBlocksPerSM / 2 : fly::kReduceBlocksPerSM;
-  const int64_t gmax = (int64_t)sm_count * (bps > 0 ? bps : 1);
+  const int64_t gmax = (int64_t)sm_count * fly::kReduceBlocksPerSM;
+  int64_t smax = n / min_units;  // pieces of at least min_units
+  if (smax > cap) smax = cap;
+  if (smax < 1) smax = 1;
   int64_t s = 0;  // > 0: every row is cut into exactly s pieces
   if (cap < 2) {
     s = 1;        // one slot per row: whole rows
   } else if (forced > 0) {
     s = forced < cap ? forced : cap;
+  } else if (inputs_ready) {
+    s = (sm_count + rows / 2) / rows;  // nearest
+    if (s > smax) s = smax;
+    if (s < 1) s = 1;
   } else {
-    int64_t G = (rows * n + min_units - 1) / min_units;
-    if (G > gmax) G = gmax;
-    if (G < 1) G = 1;
-    const int64_t Qf = (rows * n + G - 1) / G;
-    if (rows <= gmax && Qf < 8 * stride_units) {
-      // Small step: a block has only a few slices per warp, and a row boundary inside it would add one.
-      // Cut rows into whole pieces instead, as many as still fit on the device at once.
-      s = gmax / rows;
-      if (s > n / min_units) s = n / min_units;
-      if (s > cap) s = cap;
-      if (s < 1) s = 1;
-    } else {
+    s = gmax / rows;
+    if (s > smax) s = smax;
+    if (s < 1) s = 1;
+    const int64_t blocks = rows * s, waves = (blocks + gmax - 1) / gmax;
+    const bool could_fill = rows * n / min_units >= gmax;  // enough work for a full grid at all
+    if (could_fill && 4 * blocks < 3 * waves * gmax) {
+      // the last wave would be mostly empty: pack the rows end to end and cut the range evenly instead
+      s = 0;
+      const int64_t Qf = (rows * n + gmax - 1) / gmax;
       pl.Q = (Qf + 63) / 64 * 64;  // piece starts on 1 KB boundaries of the row where the row length allows
       const int64_t qmin = (n + (cap - 1) - 1) / (cap - 1);  // a row never spans more than cap blocks
       if (pl.Q < qmin) pl.Q = qmin;

@@ -93,9 +93,12 @@ def test_launch_geometry_rule():
     assert p.grid == 144 * 4 and p.slots == 4                 # small step: whole pieces, all resident (4 blocks per SM)
     assert p.row_span == 4 * p.units_per_block and p.units_per_block * 4 >= row_units
     p2 = Bd.plan(148, 144, 128256, inputs_ready=True)
-    assert p2.grid == 144 * 2                                 # overlapped steps: two grids resident together
+    assert p2.grid == 144                                     # overlapping steps: about one block per SM, several steps deep
+    assert Bd.plan(148, 16, 128256, inputs_ready=True).grid == 16 * 9
     big = Bd.plan(148, 1088, 128256)
-    assert big.row_span == row_units and big.grid <= 148 * 4 and big.grid >= 148 * 4 - 4   # large step: rows packed end to end
+    assert big.grid == 1088 and big.slots == 1                # more rows than resident slots: whole rows, two well-filled waves
+    odd = Bd.plan(148, 700, 128256)                           # 700 whole rows would leave 82 % of the second wave empty:
+    assert odd.row_span == row_units and 148 * 4 - 4 <= odd.grid <= 148 * 4   # rows packed end to end, cut evenly
     assert Bd.plan(148, 1, 128256).units_per_block >= 1024    # never less than 16 KB per block
     assert Bd.plan(148, 9, 32000, dtype="f32").grid == 9 * 7
     L = Bd.lib()
@@ -127,3 +130,5 @@ def test_launch_geometry_rule():
                         assert span % Q == 0 and span // Q <= forced
                     elif not ready:
                         assert p.grid <= max(148 * 4, rows)
+                    else:
+                        assert p.grid <= max(2 * 148, rows)
