@@ -89,36 +89,61 @@ struct FlatPlan {
   int slots = 1;
   int pieces = 0;     // > 0: every row is cut into exactly this many pieces (span = pieces * Q)
 };
-// Launch shape.  Measured on the bench workloads (144 .. 2304 rows of 250 - 300 KB): whole pieces of rows, one per
+// Launch shape.  Measured on the bench workloads (9 .. 2304 rows of 128 - 300 KB): whole pieces of rows, one per
 // block, are at least as fast as packed rows whenever they fill the resident slots reasonably well - a row boundary
 // inside a block drains that block's copy ring once, and the hardware scheduler back-fills a second wave well.
-//   plain stream order   pieces per row so that the grid just fits on the device at once (4 blocks per SM);
-//                        more rows than slots: whole rows, several waves
-//   inputs_ready         about one block per SM: consecutive steps then overlap four deep, which hides each
-//                        step's ramp and its hand-off tail behind its neighbours' streaming
+// A block's warps walk its piece in strides of `stride_units` (one slice per warp), so a piece of 3.1 strides costs
+// its slowest warp 4 slices: among the piece counts that fit, the one with the fewest slices on the busiest SM wins.
+//   plain stream order   the grid fits on the device at once (4 blocks per SM); cost = blocks on the busiest SM x
+//                        slices per warp, ties go to the count nearest two blocks per SM (the next step's blocks
+//                        can then already be resident, waiting); more rows than slots: whole rows, several waves
+//   inputs_ready         throughput, not latency: few large pieces (a quarter of a block per SM and step is
+//                        enough, consecutive steps overlap many deep), the count with the fewest slices per row
 //   packed rows          only where whole pieces would leave more than a quarter of the last wave's slots empty
+int64_t piece_units(int64_t n, int64_t s) {
+  int64_t q = (n + s - 1) / s;
+  if (s > 1) q = (q + 7) / 8 * 8;  // pieces start on 128-byte boundaries of the row
+  return q;
+}
 FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int64_t stride_units, int cap,
                    bool inputs_ready, int forced) {
-  (void)stride_units;
   FlatPlan pl;
   const int64_t gmax = (int64_t)sm_count * fly::kReduceBlocksPerSM;
   int64_t smax = n / min_units;  // pieces of at least min_units
   if (smax > cap) smax = cap;
   if (smax < 1) smax = 1;
+  auto slices = [&](int64_t s) { return (piece_units(n, s) + stride_units - 1) / stride_units; };
   int64_t s = 0;  // > 0: every row is cut into exactly s pieces
   if (cap < 2) {
     s = 1;        // one slot per row: whole rows
   } else if (forced > 0) {
     s = forced < cap ? forced : cap;
   } else if (inputs_ready) {
-    s = (sm_count + rows / 2) / rows;  // nearest
-    if (s > smax) s = smax;
-    if (s < 1) s = 1;
+    int64_t target = sm_count / (4 * rows);
+    if (target > smax) target = smax;
+    if (target < 1) target = 1;
+    int64_t best = -1;
+    for (int64_t c = 1; c <= target; ++c) {
+      const int64_t cost = c * slices(c);  // slices per row
+      if (best < 0 || cost <= best) { best = cost; s = c; }
+    }
+  } else if (rows >= gmax) {
+    s = 1;
   } else {
-    s = gmax / rows;
-    if (s > smax) s = smax;
+    int64_t best = -1, best_dist = 0;
+    for (int64_t c = 1; c <= smax && rows * c <= gmax; ++c) {
+      const int64_t cost = ((rows * c + sm_count - 1) / sm_count) * slices(c);
+      int64_t dist = rows * c - 2 * sm_count;
+      if (dist < 0) dist = -dist;
+      if (best < 0 || cost < best || (cost == best && dist < best_dist)) { best = cost; best_dist = dist; s = c; }
+    }
     if (s < 1) s = 1;
-    const int64_t blocks = rows * s, waves = (blocks + gmax - 1) / gmax;
+  }
+  if (s > 0 && cap >= 2 && forced <= 0 && !inputs_ready) {
+    int64_t s_fill = gmax / rows;  // the most pieces per row that still fit at once
+    if (s_fill > smax) s_fill = smax;
+    if (s_fill < 1) s_fill = 1;
+    const int64_t blocks = rows * s_fill, waves = (blocks + gmax - 1) / gmax;
     const bool could_fill = rows * n / min_units >= gmax;  // enough work for a full grid at all
     if (could_fill && 4 * blocks < 3 * waves * gmax) {
       // the last wave would be mostly empty: pack the rows end to end and cut the range evenly instead
@@ -132,8 +157,7 @@ FlatPlan plan_flat(int sm_count, int64_t rows, int64_t n, int64_t min_units, int
   }
   if (s > 0) {
     if (s > n) s = n;
-    pl.Q = (n + s - 1) / s;
-    if (s > 1) pl.Q = (pl.Q + 7) / 8 * 8;        // pieces start on 128-byte boundaries of the row
+    pl.Q = piece_units(n, s);
     s = (n + pl.Q - 1) / pl.Q;                   // pieces that are not empty
     pl.span = s * pl.Q;
     pl.pieces = (int)s;

@@ -90,11 +90,13 @@ def test_launch_geometry_rule():
     row_units = 128256 // 8                                   # 16-byte segments in one bf16 row of the Llama-3 vocabulary
     p = Bd.plan(148, 144, 128256)
     assert p.units_per_row == row_units
-    assert p.grid == 144 * 4 and p.slots == 4                 # small step: whole pieces, all resident (4 blocks per SM)
-    assert p.row_span == 4 * p.units_per_block and p.units_per_block * 4 >= row_units
+    assert p.grid == 144 * 2 and p.slots == 2                 # whole pieces, all resident; 1, 2 and 4 pieces cost the busiest SM
+    assert p.row_span == 2 * p.units_per_block and p.units_per_block * 2 >= row_units   # the same, 2 is nearest two blocks per SM
+    assert Bd.plan(148, 144, 128256, forced_pieces=3).grid == 144 * 3
     p2 = Bd.plan(148, 144, 128256, inputs_ready=True)
     assert p2.grid == 144                                     # overlapping steps: about one block per SM, several steps deep
-    assert Bd.plan(148, 16, 128256, inputs_ready=True).grid == 16 * 9
+    assert Bd.plan(148, 16, 128256, inputs_ready=True).grid == 16 * 2
+    assert Bd.plan(148, 16, 128256).grid == 16 * 9            # 9 pieces of 1.74 strides: two slices per warp, one block per SM
     big = Bd.plan(148, 1088, 128256)
     assert big.grid == 1088 and big.slots == 1                # more rows than resident slots: whole rows, two well-filled waves
     odd = Bd.plan(148, 700, 128256)                           # 700 whole rows would leave 82 % of the second wave empty:
