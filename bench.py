@@ -50,9 +50,9 @@ MIN_TIMED_S = 0.05                 # every timed region lasts at least this long
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
 # (bytes), keyed by kernel; None where the kernel has changed since its counters were taken.
 NCU_TRAFFIC = {
-    # reduce_rows_flat, long_draft_batch (279,085,056 algorithmic bytes): 279.15 MB read + 6.00 MB written
+    # reduce_rows_flat, long_draft_batch (279,085,056 algorithmic bytes): 279.14 MB read + 3.83 MB written
     # (profiles/reduce_rows_flat_long_draft_batch.md); scaled to other workloads by their algorithmic bytes
-    "reduce_rows_flat": {"bytes": 285.16e6, "units": 279085056},
+    "reduce_rows_flat": {"bytes": 282.97e6, "units": 279085056},
     # lmhead_verify_kernel at V = 64000: 1.0675 GB read + 4.9 MB written (profiles/lmhead_verify_kernel_fused_lm_head.md);
     # scaled by V
     "lmhead_verify_kernel": {"bytes": 1.0724e9, "units": 64000},
