@@ -469,3 +469,20 @@ def test_carried_state_that_the_library_never_writes_is_flagged_and_ignored():
     assert (flags[[1, 2, 3, 4, 5], 0] & 8).all() and not (flags[[0, 6, 7], 0] & 8).any()
     toks = out.out_tokens.cpu().numpy()
     assert toks.max() < w.V and toks.min() >= -1 and (out.rollback.cpu().numpy() >= 0).all()
+
+
+@pytest.mark.parametrize("dtype,B,K,V", [("bf16", 50, 7, 128256), ("bf16", 100, 6, 128256), ("f32", 100, 3, 32000),
+                                         ("bf16", 64, 9, 50264)])
+def test_rows_packed_end_to_end(dtype, B, K, V):
+    # row counts for which whole rows would leave most of a wave of blocks empty: the rows are laid end to end and cut
+    # into equal block ranges, so blocks start and end in the middle of rows and cover several pieces
+    from paper_2511_22972_b200 import binding as Bd
+    w = small(dtype, B=B, K=K, V=V)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    p = Bd.plan(sms, w.rows, V, dtype)
+    assert p.row_span == p.units_per_row and p.units_per_row % p.units_per_block != 0, "this shape is meant to be packed"
+    fv = FlyVerify(B, K, V, dtype)
+    logits, draft = draw(w, step=B)
+    check(fv, logits, draft, 1.0, 2, what=f"packed rows {dtype} rows={w.rows} V={V}")
+    check(fv, logits, draft, 1.0, 2, what="packed rows, scan as a kernel of its own") if fv.set_scan_mode(True) is None else None
+    fv.close()
