@@ -366,8 +366,10 @@ __device__ __forceinline__ void flush_pending(const Pending* pend, int np, int s
   if (lane < np) partials[(int64_t)pend[lane].row * slots + pend[lane].slot] = pend[lane].p;
   if (tail.tickets == nullptr) return;
   __threadfence();  // the partials written above are visible ...
-  __syncwarp();
-  __threadfence();  // ... before lane 0 takes any ticket
+  if (np > 1) {     // (one piece: lane 0 wrote it and lane 0 takes its ticket, its own fence is enough)
+    __syncwarp();
+    __threadfence();  // ... before lane 0 takes any ticket
+  }
   for (int k = 0; k < np; ++k) sequence_tail(tail, pend[k].row, pend[k].units, lane, sm_y);
 }
 

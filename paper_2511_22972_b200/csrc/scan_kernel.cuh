@@ -143,7 +143,9 @@ __device__ __forceinline__ void scan_one_sequence(const ScanParams& p, int b, in
         for (int t = 0; t < 4; ++t) merge_partial(acc, q[t], p.scale);
       }
       // entropy is non-negative; rounding may leave -1e-7 on a one-hot row
-      const float H = fmaxf(kLn2 * (log2f(acc.S) - acc.u / acc.S), 0.f);
+      // lg2.approx and the fast division are good to ~1e-6 here (S >= 1 once a row has a finite entry); this is the
+      // end of the step's critical path
+      const float H = fmaxf(kLn2 * (lg2_approx(acc.S) - __fdividef(acc.u, acc.S)), 0.f);
       uint32_t flag = 0;
       if (!(fabsf(acc.S) <= 3.0e38f) || !(acc.mx <= 3.0e38f) || acc.mx <= kMaskFloor) flag |= kFlagNonFinite;
       if (failed) flag |= kFlagStepFailed;
