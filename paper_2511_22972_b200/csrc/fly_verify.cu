@@ -20,8 +20,7 @@
 namespace {
 
 constexpr int kMaxSplits = 32;   // Partial slots per row in a handle's scratch
-// 16-byte loads per lane and slice in the row-reduction kernel (a warp keeps two slices: one in flight,
-// one being folded).
+// 16-byte copies per lane and slice in the row-reduction kernel (a warp's ring holds fly::kDepth slices).
 constexpr int kReduceUnroll = 4;
 constexpr int64_t kMinBlockBytes = 16384;   // a block that gets less than this is all fixed cost
 constexpr int kMaxK = 63;

@@ -42,7 +42,7 @@ def test_logits_path_line():
     assert "plain stream order" in d["config"]["order"]
     assert d["overlapped"]["ms_per_step"] < 1.1 * d["ms_per_step"] and d["roofline"]["frac_overlapped"] > 0
     e = d["e2e"]
-    assert e["h2d_gbs_measured"] > 1 and 0 < e["frac_of_bound"] < 1.2
+    assert e["h2d_gbs_measured"] > 1 and 0 < e["frac_of_bound"] < 1.3
 
 
 def test_default_line_carries_every_workload():
