@@ -268,11 +268,12 @@ fly_status_t fly_verify_run_static(int32_t device, int32_t vocab, fly_dtype_t lo
  * beyond fp32 rounding order.
  *
  * FLY_OPT_SPLITS          How the row reduction cuts rows into thread-block ranges.  0 (default): every row is cut
- *                         into the same number of whole pieces (at least 16 KB each) - in plain stream order as
- *                         many as still fit on the device at once, with inputs_ready about one block per SM, so
- *                         that consecutive steps overlap several deep; where whole pieces would leave most of
- *                         the last wave of blocks empty, the rows are laid end to end and that range is cut
- *                         evenly instead (a block may then cover the end of one row and the start of the next).
+ *                         into the same number of whole pieces (at least 16 KB each) - in plain stream order the
+ *                         count that keeps the grid on the device at once with the least work on the busiest SM,
+ *                         with inputs_ready few large pieces, so that consecutive steps overlap many deep; where
+ *                         whole pieces would leave most of the last wave of blocks empty, the rows are laid end
+ *                         to end and that range is cut evenly instead (a block may then cover the end of one row
+ *                         and the start of the next).
  *                         s > 0: every row is cut into exactly s pieces (1..32), one thread block each (for
  *                         tests and experiments).
  * FLY_OPT_SCAN_MODE       0 (default): the acceptance scan runs as the tail of the row-reduction
