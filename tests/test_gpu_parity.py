@@ -486,3 +486,28 @@ def test_rows_packed_end_to_end(dtype, B, K, V):
     check(fv, logits, draft, 1.0, 2, what=f"packed rows {dtype} rows={w.rows} V={V}")
     check(fv, logits, draft, 1.0, 2, what="packed rows, scan as a kernel of its own") if fv.set_scan_mode(True) is None else None
     fv.close()
+
+
+def test_two_handles_on_two_streams_at_once():
+    # a handle owns its scratch: two handles may run concurrently on two streams without disturbing each other
+    from paper_2511_22972_b200 import VerifyBuffers, verify
+    wa = small("bf16", B=16, K=8, V=128256)
+    wb = small("f32", B=7, K=5, V=32000)
+    fa, fb = FlyVerify(wa.B, wa.K, wa.V, "bf16"), FlyVerify(wb.B, wb.K, wb.V, "f32")
+    ins_a = [draw(wa, step=s) for s in range(4)]
+    ins_b = [draw(wb, step=s) for s in range(4)]
+    outs_a = [VerifyBuffers(wa.B, wa.K, DEV) for _ in ins_a]
+    outs_b = [VerifyBuffers(wb.B, wb.K, DEV) for _ in ins_b]
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for rep in range(20):
+        for (la, da), oa, (lb, db), ob in zip(ins_a, outs_a, ins_b, outs_b):
+            verify(fa, la, da, oa, theta=1.0, W=3, stream=sa.cuda_stream, inputs_ready=rep % 2 == 1)
+            verify(fb, lb, db, ob, theta=1.0, W=2, stream=sb.cuda_stream)
+    torch.cuda.synchronize()
+    for (la, da), oa in zip(ins_a, outs_a):
+        assert_parity(oa, oracle_step(la, da, 1.0, 3), "stream a")
+    for (lb, db), ob in zip(ins_b, outs_b):
+        assert_parity(ob, oracle_step(lb, db, 1.0, 2), "stream b")
+    fa.close()
+    fb.close()
