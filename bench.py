@@ -372,7 +372,7 @@ class OraclePool:
         self.share = max(1, min(-(-w.B // cores), rows_per_core // (w.K + 1)))   # sequences per worker and round
         self.workers = max(1, min(cores, w.B // self.share))
         self.ws = S.shrink(w, B=self.share)
-        ctx = mp.get_context("fork")
+        ctx = mp.get_context("forkserver")   # workers are forked from a clean server process, not from this CUDA process
         self.pool = ctx.Pool(self.workers, initializer=_pool_init, initargs=(ctx.Barrier(self.workers),))
         self.rows_per_round = self.workers * self.ws.rows
         self.w = w
