@@ -283,3 +283,37 @@ def test_flagged_position_inside_a_carried_window_revokes_it():
     r = O.verify_batch(x, np.array([[0, 0, 0]]), theta=0.0, W=1, boundary="carry", state_in=np.array([[1, 3, 2]]))
     assert r.accept_len.tolist() == [1] and r.rollback.tolist() == [3]
     assert r.out_tokens.tolist() == [[2, -1, -1, -1]] and r.state_out.tolist() == [[0, 0, -1]]
+
+
+def test_verify_batch_against_an_independent_composition_on_random_tiny_batches():
+    # End to end pin of verify_batch's plumbing (which row meets which draft, the bonus row, the threshold unit, the
+    # emitted tokens): the expected values come from a different route - the exactly rounded pure-Python row
+    # statistics (row_stats_loops) and the streaming restatement of the rule above, neither of which verify_batch uses.
+    rng = np.random.default_rng(2511)
+    for case in range(300):
+        B, K, V = int(rng.integers(1, 4)), int(rng.integers(1, 7)), int(rng.integers(2, 7))
+        W = int(rng.integers(0, K + 2))
+        unit = "nats" if case % 2 == 0 else "normalized"
+        theta = float(rng.uniform(0.05, 1.2)) if unit == "nats" else float(rng.uniform(0.05, 0.95))
+        logits = np.round(rng.normal(size=(B, K + 1, V)) * 2.5, 2)            # distinct enough: no accidental ties
+        draft = rng.integers(0, V, size=(B, K))
+        th_nats = theta if unit == "nats" else theta * math.log(V)
+        want_s, want_toks = [], []
+        skip = False
+        for b in range(B):
+            stats = [O.row_stats_loops(list(logits[b, i])) for i in range(K + 1)]
+            H = [h for h, _ in stats]
+            y = [t for _, t in stats]
+            if any(abs(h - th_nats) < 1e-9 for h in H):
+                skip = True
+            delta = [1 if int(draft[b, i]) == y[i] else 0 for i in range(K)]
+            gates = [H[i] >= th_nats for i in range(K)]
+            s = streaming_rule(delta, gates, W)
+            want_s.append(s)
+            want_toks.append([int(t) for t in draft[b, :s - 1]] + [y[s - 1]] + [-1] * (K + 1 - s))
+        if skip:
+            continue
+        got = O.verify_batch(logits, draft, theta, W, theta_unit=unit)
+        assert got.accept_len.tolist() == want_s, (case, B, K, V, W)
+        assert got.out_tokens.tolist() == want_toks, (case, B, K, V, W)
+        assert (got.row_flags == 0).all() and (got.rollback == 0).all()
