@@ -141,7 +141,8 @@ typedef struct {
    * distributions, e.g. by sampling at temperature 1.  The paper's method text defines y_i only as the
    * argmax (Eq. 1) although it reports temperature-1 results, so this is a hook, not the paper's rule:
    * the given tokens replace the argmax in the match indicator (Eq. 2) and in the emitted tokens;
-   * the entropy gate still uses the entropy of the logits.  target_argmax still reports the argmax. */
+   * the entropy gate still uses the entropy of the logits (at `temperature`).  target_argmax still reports
+   * the argmax. */
   const int32_t* target_tokens;
 
   /* Temperature T of the target distribution: the entropy of Eq. 5 is taken of softmax(l / T), the
@@ -158,8 +159,9 @@ typedef struct {
    * 1: the caller guarantees that the logits and draft tokens of this step were complete BEFORE the
    *    previous kernel in the stream was launched (e.g. a queue of steps over inputs that are already in
    *    memory).  The kernel then starts READING at once, next to the draining previous kernel, and waits
-   *    only before its first write.  Wrong results if the guarantee does not hold - in a decode loop, where
-   *    the previous kernel produces this step's logits, leave it 0. */
+   *    only before its first write.  (state_in is read after that wait: it may be the previous step's
+   *    state_out.)  Wrong results if the guarantee does not hold - in a decode loop, where the previous
+   *    kernel produces this step's logits, leave it 0. */
   int32_t inputs_ready;
 } fly_verify_args_t;
 
